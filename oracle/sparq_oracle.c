@@ -1,0 +1,291 @@
+/*
+ * CPU oracle for the SPARQ hot path (arXiv 2105.11010) -- TEST INFRASTRUCTURE.
+ *
+ * A plain, slow, byte-at-a-time restatement of what the paper defines.  It is
+ * only ever called by the tests, by the smoke check and by the CPU-baseline
+ * leg of the benchmark; the CUDA library shares no code with it and never
+ * calls it.  There is no blocking, fusion or reordering here beyond the
+ * definitions: rows are independent, and the only concession to run time is
+ * an OpenMP loop over independent output rows.
+ *
+ * Conventions
+ *   n     window width in bits (the paper uses 4, 3 and 2; Section 3.1, 5.1).
+ *   mask  placement set: bit s set <=> the window may sit at bits [s+n-1 : s],
+ *         i.e. be followed by a shift-left of s (Section 3.1: 5opt = shifts
+ *         {0,1,2,3,4}, 3opt = {0,2,4}, 2opt = {0,4}).
+ *   rnd   0 = trim the bits below the window, 1 = round on the residual LSBs
+ *         (Section 3.1, last paragraph).  The paper does not say which way a
+ *         tie goes: ties go UP here (add half, then trim).  PARITY UNPINNED
+ *         for the tie direction alone; everything else is pinned by the tests.
+ *   mode  0 = none (plain 8b-8b), 1 = bSPARQ on every activation,
+ *         2 = vSPARQ on adjacent pairs with bSPARQ when both are non-zero (Eq. 2).
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---- Section 3.1: bSPARQ ------------------------------------------------ */
+
+/* Index of the most significant set bit of a non-zero byte ("searching for the
+ * first most significant toggled bit", Section 3.1). */
+static int leading_one(unsigned x)
+{
+    int p = 7;
+    while (p > 0 && !((x >> p) & 1u)) --p;
+    return p;
+}
+
+/* The placement actually used for x: the lowest allowed shift whose n-bit window
+ * still covers the leading one (Section 3.1 examples: 27 -> [4:1] under 5opt,
+ * [5:2] under 3opt, [7:4] under 2opt).  Returns -1 if the set has no such shift. */
+int oracle_window_shift(unsigned x, int n, unsigned mask)
+{
+    if (x == 0) return 0;
+    int p = leading_one(x);
+    for (int s = 0; s <= 8 - n; ++s) {
+        if (!((mask >> s) & 1u)) continue;
+        if (s + n - 1 >= p) return s;
+    }
+    return -1;
+}
+
+/* Is v exactly "an n-bit window shifted left by an allowed amount"? */
+static int representable(unsigned v, int n, unsigned mask)
+{
+    for (int s = 0; s <= 8 - n; ++s) {
+        if (!((mask >> s) & 1u)) continue;
+        if ((v >> s) < (1u << n) && (v & ((1u << s) - 1u)) == 0) return 1;
+    }
+    return 0;
+}
+
+/* bSPARQ of one 8-bit activation (Section 3.1).  n = 8 is the identity. */
+unsigned oracle_bsparq(unsigned x, int n, unsigned mask, int rnd)
+{
+    x &= 0xFFu;
+    if (x == 0 || n >= 8) return x;
+    int s = oracle_window_shift(x, n, mask);
+    if (s < 0) return 0xFFFFFFFFu; /* invalid placement set */
+    if (!rnd) return (x >> s) << s;                /* trim */
+    unsigned half = s ? (1u << (s - 1)) : 0u;
+    unsigned r = (x + half) >> s;                  /* round on the residual LSBs, ties up */
+    if (r < (1u << n)) return r << s;
+    /* The window overflowed to 2^n: the value is the single bit 2^(s+n).  It is
+     * kept when a higher placement can hold it; at the top of the 8-bit range it
+     * cannot, and the window saturates. */
+    unsigned v = 1u << (s + n);
+    if (v <= 255u && representable(v, n, mask)) return v;
+    return ((1u << n) - 1u) << s;
+}
+
+/* The window bits themselves (before the shift-left), for the paper's examples. */
+unsigned oracle_bsparq_window(unsigned x, int n, unsigned mask, int rnd, int *shift_out)
+{
+    unsigned q = oracle_bsparq(x, n, mask, rnd);
+    int s = 0;
+    /* the placement of the RESULT: lowest allowed shift that represents q */
+    for (s = 0; s <= 8 - n; ++s) {
+        if (!((mask >> s) & 1u)) continue;
+        if ((q >> s) < (1u << n) && (q & ((1u << s) - 1u)) == 0) break;
+    }
+    if (!rnd) s = oracle_window_shift(x, n, mask); /* trim never moves the window */
+    if (shift_out) *shift_out = s;
+    return q >> s;
+}
+
+/* ---- Section 3.2: vSPARQ ------------------------------------------------ */
+
+/* A lone non-zero activation of a pair owns the whole 2n-bit budget (Section 1,
+ * contributions; Section 5.1: "total window sizes are 6 and 4 bits" for n = 3, 2).
+ * With 2n >= 8 that is the exact 8-bit value.  Otherwise it is a 2n-bit window made
+ * of the two adjacent n-bit halves of Eq. 4, which may sit at any shift 0..8-2n. */
+static unsigned lone_budget(unsigned x, int n, int rnd)
+{
+    int wide = 2 * n;
+    if (wide >= 8) return x & 0xFFu;
+    unsigned full = (1u << (8 - wide + 1)) - 1u; /* shifts 0 .. 8-2n, all allowed */
+    return oracle_bsparq(x, wide, full, rnd);
+}
+
+/* Eq. 2: the pair (a, b) of adjacent activations along the reduction dimension. */
+void oracle_vsparq_pair(unsigned a, unsigned b, int n, unsigned mask, int rnd,
+                        unsigned *qa, unsigned *qb)
+{
+    a &= 0xFFu; b &= 0xFFu;
+    if (b == 0)      { *qa = lone_budget(a, n, rnd); *qb = 0; }
+    else if (a == 0) { *qa = 0; *qb = lone_budget(b, n, rnd); }
+    else             { *qa = oracle_bsparq(a, n, mask, rnd); *qb = oracle_bsparq(b, n, mask, rnd); }
+}
+
+/* The activation transform T over `rows` rows of `row_len` bytes.  Pairs are
+ * (2j, 2j+1) inside a row (Eq. 1) and never cross rows; an odd row length leaves
+ * the last element paired with an implicit zero. */
+void oracle_transform(const uint8_t *in, uint8_t *out, size_t rows, size_t row_len,
+                      int mode, int n, unsigned mask, int rnd)
+{
+    for (size_t r = 0; r < rows; ++r) {
+        const uint8_t *x = in + r * row_len;
+        uint8_t *y = out + r * row_len;
+        if (mode == 0) {
+            for (size_t k = 0; k < row_len; ++k) y[k] = x[k];
+        } else if (mode == 1) {
+            for (size_t k = 0; k < row_len; ++k) y[k] = (uint8_t)oracle_bsparq(x[k], n, mask, rnd);
+        } else {
+            for (size_t k = 0; k < row_len; k += 2) {
+                unsigned a = x[k], b = (k + 1 < row_len) ? x[k + 1] : 0u, qa, qb;
+                oracle_vsparq_pair(a, b, n, mask, rnd, &qa, &qb);
+                y[k] = (uint8_t)qa;
+                if (k + 1 < row_len) y[k + 1] = (uint8_t)qb;
+            }
+        }
+    }
+}
+
+/* ---- Eq. 1: the dot product over the transformed activations ------------- */
+
+/* acc[m][j] = sum_k T(A)[m][k] * B[k][j]; A is M x K (row-major, u8), B is the
+ * logical K x N matrix (row-major, s8), int32 accumulation.  |acc| <= K*255*128,
+ * which cannot overflow 32 bits for K <= 65793. */
+void oracle_gemm(const uint8_t *A, const int8_t *B, int32_t *acc,
+                 int64_t M, int64_t N, int64_t K,
+                 int mode, int n, unsigned mask, int rnd)
+{
+#pragma omp parallel
+    {
+        uint8_t *ta = (uint8_t *)__builtin_malloc((size_t)(K > 0 ? K : 1));
+#pragma omp for schedule(static)
+        for (int64_t m = 0; m < M; ++m) {
+            oracle_transform(A + m * K, ta, 1, (size_t)K, mode, n, mask, rnd);
+            for (int64_t j = 0; j < N; ++j) acc[m * N + j] = 0;
+            for (int64_t k = 0; k < K; ++k) {
+                int32_t a = ta[k];
+                const int8_t *brow = B + k * N;
+                for (int64_t j = 0; j < N; ++j) acc[m * N + j] += a * (int32_t)brow[j];
+            }
+        }
+        __builtin_free(ta);
+    }
+}
+
+/* Same product accumulated in 64 bits (tiny shapes only): equality with the int32
+ * result shows that the 32-bit accumulator never wrapped. */
+void oracle_gemm_i64(const uint8_t *A, const int8_t *B, int64_t *acc,
+                     int64_t M, int64_t N, int64_t K,
+                     int mode, int n, unsigned mask, int rnd)
+{
+    uint8_t *ta = (uint8_t *)__builtin_malloc((size_t)(K > 0 ? K : 1));
+    for (int64_t m = 0; m < M; ++m) {
+        oracle_transform(A + m * K, ta, 1, (size_t)K, mode, n, mask, rnd);
+        for (int64_t j = 0; j < N; ++j) {
+            int64_t s = 0;
+            for (int64_t k = 0; k < K; ++k) s += (int64_t)ta[k] * (int64_t)B[k * N + j];
+            acc[m * N + j] = s;
+        }
+    }
+    __builtin_free(ta);
+}
+
+/* ---- Section 4: convolution as the same dot product --------------------- */
+
+/* Direct convolution.  x is NHWC u8, w is [cout][r][s][c] s8, dilation 1.  The
+ * reduction runs over (r, s, c) with c fastest, so vSPARQ pairs are adjacent input
+ * channels of one pixel; T is therefore applied once to the whole input tensor with
+ * rows = pixels.  Taps that fall outside the image contribute nothing.
+ *
+ * Only the output pixels listed in `pix` (linear index over n, ho, wo) are computed
+ * when pix != NULL; otherwise all of them.  acc is [npix][cout]. */
+void oracle_conv2d_nhwc(const uint8_t *x, int nb, int h, int w, int c,
+                        const int8_t *wgt, int cout, int r, int s,
+                        int stride_h, int stride_w, int pad_h, int pad_w,
+                        int mode, int n, unsigned mask, int rnd,
+                        const int64_t *pix, int64_t npix, int32_t *acc)
+{
+    int ho = (h + 2 * pad_h - r) / stride_h + 1;
+    int wo = (w + 2 * pad_w - s) / stride_w + 1;
+    int64_t total = (int64_t)nb * ho * wo;
+    int64_t count = pix ? npix : total;
+    size_t in_pixels = (size_t)nb * h * w;
+    uint8_t *tx = (uint8_t *)__builtin_malloc(in_pixels * (size_t)c + 1);
+    oracle_transform(x, tx, in_pixels, (size_t)c, mode, n, mask, rnd);
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < count; ++i) {
+        int64_t p = pix ? pix[i] : i;
+        int img = (int)(p / ((int64_t)ho * wo));
+        int oy = (int)((p / wo) % ho);
+        int ox = (int)(p % wo);
+        for (int co = 0; co < cout; ++co) {
+            int32_t sum = 0;
+            for (int fr = 0; fr < r; ++fr) {
+                int iy = oy * stride_h - pad_h + fr;
+                if (iy < 0 || iy >= h) continue;
+                for (int fs = 0; fs < s; ++fs) {
+                    int ix = ox * stride_w - pad_w + fs;
+                    if (ix < 0 || ix >= w) continue;
+                    const uint8_t *xp = tx + (((size_t)img * h + iy) * w + ix) * (size_t)c;
+                    const int8_t *wp = wgt + (((size_t)co * r + fr) * s + fs) * (size_t)c;
+                    for (int ci = 0; ci < c; ++ci) sum += (int32_t)xp[ci] * (int32_t)wp[ci];
+                }
+            }
+            acc[i * cout + co] = sum;
+        }
+    }
+    __builtin_free(tx);
+}
+
+/* ---- Dequantize, bias, ReLU, requantize ---------------------------------- */
+
+/* The paper only fixes the quantization scheme (Section 5: per-layer activation
+ * scale, per-kernel weight scale); the arithmetic below is this library's stated
+ * fp32 sequence, one IEEE operation per line, no contraction:
+ *     t = (float)acc                       int32 -> fp32, round to nearest even
+ *     y = fma(t, scale[j], bias[j])        single rounding
+ *     y = relu ? max(y, 0) : y             (y > 0 ? y : 0)
+ *     z = y * inv_out_scale
+ *     u = rint(z)                          nearest even
+ *     q = clamp(u, 0, 255) as uint8        NaN -> 0
+ * Any of f32_out / u8_out may be NULL. */
+void oracle_epilogue(const int32_t *acc, int64_t M, int64_t N,
+                     const float *scale, const float *bias, int relu, float inv_out_scale,
+                     float *f32_out, uint8_t *u8_out)
+{
+    for (int64_t m = 0; m < M; ++m) {
+        for (int64_t j = 0; j < N; ++j) {
+            volatile float t = (float)acc[m * N + j];
+            volatile float y = fmaf(t, scale[j], bias ? bias[j] : 0.0f);
+            if (relu) y = (y > 0.0f) ? y : 0.0f;
+            if (f32_out) f32_out[m * N + j] = y;
+            if (u8_out) {
+                volatile float z = y * inv_out_scale;
+                volatile float u = rintf(z);
+                uint8_t q;
+                if (!(u > 0.0f)) q = 0;             /* negative, zero and NaN */
+                else if (u > 255.0f) q = 255;
+                else q = (uint8_t)u;
+                u8_out[m * N + j] = q;
+            }
+        }
+    }
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void oracle_set_num_threads(int t)
+{
+#ifdef _OPENMP
+    if (t > 0) omp_set_num_threads(t);
+#else
+    (void)t;
+#endif
+}
