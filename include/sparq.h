@@ -1,0 +1,150 @@
+/*
+ * sparq.h -- C ABI of the B200 (sm_100a) SPARQ library.
+ *
+ * SPARQ (arXiv 2105.11010, "Post-Training Sparsity-Aware Quantization") trims
+ * already-quantized unsigned 8-bit activations to an n-bit window that starts at the
+ * leading one (bSPARQ, Section 3.1) and lets a lone non-zero activation of an adjacent
+ * pair keep the 2n-bit budget of the pair (vSPARQ, Section 3.2, Eq. 2).  The trimmed
+ * value is still an 8-bit integer (window << shift), so the dot product of Eq. 1 is an
+ * ordinary u8 x s8 -> s32 contraction over the transformed activations.
+ *
+ * Conventions common to all entry points
+ *   - Unless a parameter says HOST, every data pointer is a DEVICE pointer that the
+ *     caller owns; the library neither frees nor keeps it after the enqueued work ends.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  A call
+ *     validates its arguments on the host, enqueues its kernels on `stream` and returns
+ *     without synchronizing.
+ *   - Return value: SPARQ_OK (0) or a negative sparq_status.  On error nothing has been
+ *     enqueued and sparq_last_error() describes the reason.  No entry point throws,
+ *     aborts or traps the device.
+ *   - The library is thread-compatible: concurrent calls are allowed, the error string
+ *     is per host thread.
+ */
+#ifndef SPARQ_H_
+#define SPARQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SPARQ_API __attribute__((visibility("default")))
+#else
+#define SPARQ_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SPARQ_OK = 0,
+    SPARQ_ERR_INVALID_ARG = -1, /* null pointer, negative size, bad mode / width / placement set */
+    SPARQ_ERR_UNSUPPORTED = -2, /* a shape or alignment this build has no kernel for */
+    SPARQ_ERR_CUDA = -3,        /* a CUDA runtime / driver call failed (text in sparq_last_error) */
+    SPARQ_ERR_TIMEOUT = -4      /* a bounded device-side wait expired (reported by sparq_check) */
+} sparq_status;
+
+enum { SPARQ_MODE_NONE = 0, SPARQ_MODE_BSPARQ = 1, SPARQ_MODE_VSPARQ = 2 };
+enum { SPARQ_ROUND_TRUNCATE = 0, SPARQ_ROUND_NEAREST = 1 };
+
+/* Named placement sets: bit s set <=> the window may occupy bits [s+n-1 : s], i.e. be
+ * shifted left by s.  Section 3.1 (5opt/3opt/2opt, n = 4); Section 5.1 (6opt n = 3,
+ * 7opt n = 2). */
+#define SPARQ_SET_5OPT 0x1Fu
+#define SPARQ_SET_3OPT 0x15u
+#define SPARQ_SET_2OPT 0x11u
+#define SPARQ_SET_6OPT 0x3Fu
+#define SPARQ_SET_7OPT 0x7Fu
+
+/* The activation transform.
+ *   mode            NONE: activations are used as they are (plain A8W8).
+ *                   BSPARQ: every activation is trimmed on its own (Section 3.1; the
+ *                   "-vS" columns of Tables 2, 4 and 5).
+ *                   VSPARQ: activations are taken in pairs (2j, 2j+1) along the reduction
+ *                   axis; if one is zero the other keeps a 2n-bit window (all 8 bits when
+ *                   n = 4), otherwise both are trimmed by bSPARQ (Eq. 2).
+ *   window_bits     n = 2, 3 or 4.
+ *   placement_mask  allowed shifts; must contain 0 and 8-n, have no bit above 8-n and no
+ *                   gap between consecutive shifts wider than n.
+ *   rounding        TRUNCATE drops the bits below the window ("Trim"); NEAREST adds half a
+ *                   window LSB first ("+R"; ties go up; the top of the 8-bit range
+ *                   saturates to the all-ones window at the highest placement).
+ * With mode NONE the other three fields are ignored. */
+typedef struct {
+    int32_t mode;
+    int32_t window_bits;
+    uint32_t placement_mask;
+    int32_t rounding;
+} sparq_params;
+
+/* What happens to the int32 accumulators (not in the paper beyond its quantization
+ * scheme, Section 5: per-layer activation scale times per-kernel weight scale).  For
+ * output column j, in fp32 and in this order, one IEEE operation each:
+ *     t = (float)acc;  y = fma(t, scale[j], bias ? bias[j] : 0);  if (relu) y = y > 0 ? y : 0;
+ *     f32_out = y;     u8_out = clamp(rint(y * inv_out_scale), 0, 255)   (NaN -> 0)
+ * Each output pointer may be NULL (that output is not produced); at least one must be
+ * non-NULL.  Outputs are M x N row-major with leading dimension N (= NHWC for the
+ * convolution).  scale may be NULL only if f32_out and u8_out are both NULL. */
+typedef struct {
+    const float *scale;   /* [N] device */
+    const float *bias;    /* [N] device, or NULL */
+    int32_t relu;         /* 0 / 1 */
+    float inv_out_scale;  /* multiplier onto the next layer's u8 grid */
+    int32_t *acc_out;     /* raw accumulators, or NULL */
+    float *f32_out;       /* dequantized fp32, or NULL */
+    uint8_t *u8_out;      /* requantized activations for the next layer, or NULL */
+} sparq_epilogue;
+
+/* Standalone transform (Sections 3.1-3.2): out[r][k] = T(in[r][:])[k] for `rows` rows of
+ * `row_len` bytes, rows stored back to back.  Pairs are (2j, 2j+1) inside a row and never
+ * cross rows; an odd row_len pairs the last element with an implicit zero.  `out` may be
+ * the same buffer as `in` (in place) but must not partially overlap it.  Any alignment is
+ * accepted; 16-byte aligned buffers with an even row_len take the fast vector path.
+ * rows == 0 or row_len == 0 is a no-op. */
+SPARQ_API int sparq_quantize(const uint8_t *in, uint8_t *out, size_t rows, size_t row_len,
+                   const sparq_params *p, void *stream);
+
+/* Fused dot products (Eq. 1 with Eq. 2 applied on the fly):
+ *     acc[m][j] = sum_k T(A)[m][k] * B[j][k]        u8 x s8 -> s32
+ * A is M x K with leading dimension lda (K contiguous); vSPARQ pairs are (2j, 2j+1) along
+ * K.  B is N x K with leading dimension ldb (K contiguous: one row per output column,
+ * which is the layout of convolution weights [cout][r][s][cin]).  The result goes through
+ * the epilogue `e`.
+ * Requirements (else SPARQ_ERR_UNSUPPORTED): A and B 16-byte aligned, lda and ldb
+ * multiples of 16, K a multiple of 16 and at most 65536; M, N >= 1 (M == 0 or N == 0 is a
+ * no-op that returns SPARQ_OK). */
+SPARQ_API int sparq_gemm_s8(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                  int64_t M, int64_t N, int64_t K,
+                  const sparq_params *p, const sparq_epilogue *e, void *stream);
+
+/* Fused convolution (Section 4: the convolution mapped onto the same dot product, here
+ * without materializing im2col).  x is NHWC u8 [n][h][w][c]; wgt is s8 [cout][r][s][c];
+ * dilation 1.  The reduction runs over (r, s, c) with c fastest, so vSPARQ pairs are
+ * adjacent input channels of one pixel, and taps outside the image contribute zero.
+ * Output pixel (img, ho, wo) is row (img*Ho + ho)*Wo + wo of the M x cout outputs, with
+ * Ho = (h + 2*pad_h - r)/stride_h + 1 and Wo likewise.
+ * Requirements (else SPARQ_ERR_UNSUPPORTED): x and wgt 16-byte aligned, c a multiple of
+ * 16 (64 or a multiple of 128 when r*s > 1), r, s in 1..7, strides in 1..8,
+ * pads < filter size. */
+SPARQ_API int sparq_conv2d_nhwc_s8(const uint8_t *x, int n, int h, int w, int c,
+                         const int8_t *wgt, int cout, int r, int s,
+                         int stride_h, int stride_w, int pad_h, int pad_w,
+                         const sparq_params *p, const sparq_epilogue *e, void *stream);
+
+/* Synchronizes `stream` and reports what the device-side code recorded since the last
+ * check: SPARQ_OK, SPARQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up (its
+ * outputs are then undefined), or SPARQ_ERR_CUDA if the stream is in error. */
+SPARQ_API int sparq_check(void *stream);
+
+/* Text of the calling thread's most recent error ("" if none).  The pointer stays valid
+ * until the thread's next failing call. */
+SPARQ_API const char *sparq_last_error(void);
+
+/* Releases what the library itself holds on the current device (cached descriptors, the
+ * status word).  Safe to call more than once; later calls re-create what they need. */
+SPARQ_API int sparq_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARQ_H_ */

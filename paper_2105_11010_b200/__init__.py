@@ -1,0 +1,17 @@
+"""B200 (sm_100a) SPARQ hot path: thin Python binding over the C-ABI library.
+
+Every step of the path runs in the library's CUDA kernels; this package only
+marshals arguments (torch tensors are used for device memory and streams).
+There is no CPU fallback: importing the binding without the built shared
+library raises.
+"""
+from ._binding import (  # noqa: F401
+    SparqParams,
+    SparqError,
+    MODE_NONE, MODE_BSPARQ, MODE_VSPARQ,
+    ROUND_TRUNCATE, ROUND_NEAREST,
+    SET_5OPT, SET_3OPT, SET_2OPT, SET_6OPT, SET_7OPT,
+    library_path, load_library,
+    sparq_quantize, sparq_gemm_s8, sparq_conv2d_nhwc_s8,
+    sparq_check, sparq_last_error, sparq_shutdown,
+)

@@ -1,0 +1,187 @@
+"""ctypes binding with the same names as the C ABI in ``include/sparq.h``.
+
+Argument marshalling only.  Tensors must already live on the CUDA device (the
+raw ``data_ptr`` is handed to the library) and work is enqueued on torch's
+current stream unless a stream is given.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+MODE_NONE, MODE_BSPARQ, MODE_VSPARQ = 0, 1, 2
+ROUND_TRUNCATE, ROUND_NEAREST = 0, 1
+SET_5OPT, SET_3OPT, SET_2OPT, SET_6OPT, SET_7OPT = 0x1F, 0x15, 0x11, 0x3F, 0x7F
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libsparq_b200.so")
+
+
+class SparqError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"sparq error {code}: {text}")
+        self.code = code
+
+
+class _CParams(ctypes.Structure):
+    _fields_ = [("mode", ctypes.c_int32), ("window_bits", ctypes.c_int32),
+                ("placement_mask", ctypes.c_uint32), ("rounding", ctypes.c_int32)]
+
+
+class _CEpilogue(ctypes.Structure):
+    _fields_ = [("scale", ctypes.c_void_p), ("bias", ctypes.c_void_p),
+                ("relu", ctypes.c_int32), ("inv_out_scale", ctypes.c_float),
+                ("acc_out", ctypes.c_void_p), ("f32_out", ctypes.c_void_p),
+                ("u8_out", ctypes.c_void_p)]
+
+
+@dataclass(frozen=True)
+class SparqParams:
+    """Mirror of ``sparq_params``."""
+    mode: int = MODE_VSPARQ
+    window_bits: int = 4
+    placement_mask: int = SET_5OPT
+    rounding: int = ROUND_NEAREST
+
+    def _c(self) -> _CParams:
+        return _CParams(self.mode, self.window_bits, self.placement_mask, self.rounding)
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the built C-ABI library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2105_11010_b200.build` "
+                "(needs nvcc); this package has no CPU fallback")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
+        L.sparq_quantize.argtypes = [vp, vp, sz, sz, ctypes.POINTER(_CParams), vp]
+        L.sparq_quantize.restype = i32
+        L.sparq_gemm_s8.argtypes = [vp, i64, vp, i64, i64, i64, i64,
+                                    ctypes.POINTER(_CParams), ctypes.POINTER(_CEpilogue), vp]
+        L.sparq_gemm_s8.restype = i32
+        L.sparq_conv2d_nhwc_s8.argtypes = [vp, i32, i32, i32, i32, vp, i32, i32, i32,
+                                           i32, i32, i32, i32,
+                                           ctypes.POINTER(_CParams), ctypes.POINTER(_CEpilogue), vp]
+        L.sparq_conv2d_nhwc_s8.restype = i32
+        L.sparq_check.argtypes = [vp]
+        L.sparq_check.restype = i32
+        L.sparq_last_error.argtypes = []
+        L.sparq_last_error.restype = ctypes.c_char_p
+        L.sparq_shutdown.argtypes = []
+        L.sparq_shutdown.restype = i32
+        _lib = L
+    return _lib
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def _dev(t: Optional[torch.Tensor], dtype, name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise ValueError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t.data_ptr() or None
+
+
+def _raise(code: int) -> None:
+    if code != 0:
+        raise SparqError(code, sparq_last_error())
+
+
+def sparq_last_error() -> str:
+    return load_library().sparq_last_error().decode()
+
+
+def sparq_check(stream=None) -> None:
+    _raise(load_library().sparq_check(_stream_ptr(stream)))
+
+
+def sparq_shutdown() -> None:
+    _raise(load_library().sparq_shutdown())
+
+
+def sparq_quantize(inp: torch.Tensor, out: torch.Tensor, rows: int, row_len: int,
+                   params: SparqParams, stream=None) -> None:
+    """``out = T(inp)`` for ``rows`` rows of ``row_len`` uint8 activations."""
+    if inp.numel() < rows * row_len or out.numel() < rows * row_len:
+        raise ValueError("tensor smaller than rows * row_len")
+    p = params._c()
+    _raise(load_library().sparq_quantize(_dev(inp, torch.uint8, "inp"), _dev(out, torch.uint8, "out"),
+                                         rows, row_len, ctypes.byref(p), _stream_ptr(stream)))
+
+
+def _epilogue(n_cols: int, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out) -> _CEpilogue:
+    for name, t in (("scale", scale), ("bias", bias)):
+        if t is not None and t.numel() < n_cols:
+            raise ValueError(f"{name} has fewer than N elements")
+    return _CEpilogue(_dev(scale, torch.float32, "scale"), _dev(bias, torch.float32, "bias"),
+                      int(bool(relu)), float(inv_out_scale),
+                      _dev(acc_out, torch.int32, "acc_out"), _dev(f32_out, torch.float32, "f32_out"),
+                      _dev(u8_out, torch.uint8, "u8_out"))
+
+
+def sparq_gemm_s8(A: torch.Tensor, B: torch.Tensor, params: SparqParams, *,
+                  scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                  relu: bool = False, inv_out_scale: float = 1.0,
+                  acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
+                  u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """``acc = T(A) @ B^T`` with A (M, K) uint8 and B (N, K) int8, then the epilogue."""
+    M, K = A.shape
+    N, K2 = B.shape
+    if K != K2:
+        raise ValueError("A and B disagree on K")
+    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out)):
+        if t is not None and t.numel() < M * N:
+            raise ValueError(f"{name} has fewer than M*N elements")
+    p = params._c()
+    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out)
+    _raise(load_library().sparq_gemm_s8(_dev(A, torch.uint8, "A"), K, _dev(B, torch.int8, "B"), K,
+                                        M, N, K, ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))
+
+
+def sparq_conv2d_nhwc_s8(x: torch.Tensor, w: torch.Tensor, stride, pad, params: SparqParams, *,
+                         scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                         relu: bool = False, inv_out_scale: float = 1.0,
+                         acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
+                         u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Fused convolution of NHWC uint8 ``x`` with [cout][r][s][c] int8 ``w``."""
+    nb, h, wd, c = x.shape
+    cout, r, s, c2 = w.shape
+    if c != c2:
+        raise ValueError("x and w disagree on the channel count")
+    ho = (h + 2 * pad[0] - r) // stride[0] + 1
+    wo = (wd + 2 * pad[1] - s) // stride[1] + 1
+    m = nb * ho * wo
+    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out)):
+        if t is not None and t.numel() < m * cout:
+            raise ValueError(f"{name} has fewer than N*Ho*Wo*Cout elements")
+    p = params._c()
+    e = _epilogue(cout, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out)
+    _raise(load_library().sparq_conv2d_nhwc_s8(_dev(x, torch.uint8, "x"), nb, h, wd, c,
+                                               _dev(w, torch.int8, "w"), cout, r, s,
+                                               stride[0], stride[1], pad[0], pad[1],
+                                               ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))

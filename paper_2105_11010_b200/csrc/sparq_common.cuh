@@ -1,0 +1,106 @@
+// Shared host/device pieces of the SPARQ library: error reporting, parameter
+// validation, and the packed (4 activations per 32-bit word) form of the
+// bSPARQ / vSPARQ transform used by both the standalone kernel and the fused GEMM.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sparq.h"
+
+namespace sparq {
+
+// ---- host side ---------------------------------------------------------------------
+
+int set_error(int code, const char *fmt, ...);
+int cuda_error(cudaError_t e, const char *what);
+
+// Host-validated, kernel-ready description of the transform.
+struct XformArgs {
+    int mode;           // SPARQ_MODE_*
+    int n;              // window bits: 2, 3, 4
+    int rnd;            // 0 trim, 1 nearest
+    int widen_rounds;   // longest run of consecutive disallowed shifts
+    uint32_t widen_c;   // per byte: bit d set for every disallowed shift d (0 < d < 8-n)
+    uint32_t mask;      // placement mask as given
+};
+
+// Checks `p` (Section 3.1 placement sets, Section 5.1 widths) and fills `x`.
+int validate_params(const sparq_params *p, XformArgs *x);
+
+// Device status word shared by all kernels of this library on the current device.
+// Bit 0: a bounded wait expired.  Allocated on first use, freed by sparq_shutdown().
+int get_status_word(unsigned int **dptr);
+
+// ---- device side -------------------------------------------------------------------
+
+#define SPARQ_HD __host__ __device__ __forceinline__
+
+// prmt.b32: byte i of the result is byte (sel nibble i & 7) of {b:a}; nibble bit 3 asks
+// for that byte's top bit replicated over all eight bits instead.
+SPARQ_HD uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+#ifdef __CUDA_ARCH__
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+#else
+    uint64_t src = ((uint64_t)b << 32) | a;
+    uint32_t d = 0;
+    for (int i = 0; i < 4; ++i) {
+        uint32_t nib = (sel >> (4 * i)) & 0xFu;
+        uint32_t byte = (uint32_t)(src >> (8 * (nib & 7u))) & 0xFFu;
+        if (nib & 8u) byte = (byte & 0x80u) ? 0xFFu : 0u;
+        d |= byte << (8 * i);
+    }
+    return d;
+#endif
+}
+
+// Mask of the bits BELOW the window for each of the four bytes of x (Section 3.1: the
+// window's top bit is the leading one, or the window sits at the bottom).  W = window
+// width.  widen_c / rounds move a window that landed on a disallowed placement up to
+// the next allowed one.
+template <int W>
+SPARQ_HD uint32_t drop_mask(uint32_t x, uint32_t widen_c, int rounds)
+{
+    constexpr uint32_t LOW = 0x01010101u * (0xFFu >> W);
+    uint32_t m = (x >> W) & LOW;                 // bits of x above the lowest window
+    m |= (m >> 1) & 0x7F7F7F7Fu;                 // smear the leading one downwards
+    if (8 - W > 2) m |= (m >> 2) & 0x3F3F3F3Fu;
+    if (8 - W > 4) m |= (m >> 4) & 0x0F0F0F0Fu;
+    for (int r = 0; r < rounds; ++r) m |= (m << 1) & widen_c;
+    return m;
+}
+
+// Trim or round four bytes given their drop masks.  Rounding adds half a window LSB;
+// a byte that would overflow 8 bits (only possible at the highest placement, where the
+// half is 0x80 >> W) keeps its trimmed value, i.e. saturates to the all-ones window.
+template <int W, bool RND>
+SPARQ_HD uint32_t apply_mask(uint32_t x, uint32_t m)
+{
+    if (!RND) return x & ~m;
+    uint32_t half = m ^ ((m >> 1) & 0x7F7F7F7Fu);   // (m + 1) >> 1 per byte
+    uint32_t x7 = x & 0x7F7F7F7Fu, x8 = x & 0x80808080u;
+    uint32_t lo = x7 + half;                        // no carry leaves a byte
+    uint32_t ovf = lo & x8;                         // bit 7: x + half >= 256
+    lo -= ovf >> W;
+    return (lo ^ x8) & ~m;
+}
+
+// T on four packed activations (bytes 0,1 and bytes 2,3 are the pairs of Eq. 2).
+template <int MODE, int N, bool RND>
+SPARQ_HD uint32_t xform_word(uint32_t x, uint32_t widen_c, int rounds)
+{
+    if (MODE == SPARQ_MODE_NONE) return x;
+    uint32_t q = apply_mask<N, RND>(x, drop_mask<N>(x, widen_c, rounds));
+    if (MODE == SPARQ_MODE_BSPARQ) return q;
+    // vSPARQ: a byte whose partner is zero keeps the 2n-bit budget.
+    uint32_t lone = x;
+    if (2 * N < 8) lone = apply_mask<2 * N, RND>(x, drop_mask<(2 * N < 8 ? 2 * N : 4)>(x, 0u, 0));
+    uint32_t nz = ((x & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | x;   // bit 7 of each byte: byte != 0
+    uint32_t partner_nz = prmt(nz, nz, 0xAB89u);           // swap within pairs, replicate bit 7
+    return (q & partner_nz) | (lone & ~partner_nz);
+}
+
+}  // namespace sparq
