@@ -92,7 +92,8 @@ def test_full_size_2_30_sampled(mode):
         want = oracle.transform(x[s:s + win].reshape(-1, row_len), mode, 4, 0x1F, 1).reshape(-1)
         assert np.array_equal(got, want), s
     # properties that hold at any size, checked on the whole tensor on the device
-    assert int((yd > xd + 8).sum()) == 0                     # never more than half a top-window LSB up
+    diff = yd.to(torch.int16) - xd.to(torch.int16)
+    assert int(diff.max()) <= 8 and int(diff.min()) >= -8    # within half a top-window LSB
     assert bool(((xd == 0) == (yd == 0)).all())              # zeros, and only zeros, map to zero
     small = xd < 16
     assert bool((yd[small] == xd[small]).all())              # values below 16 unchanged
