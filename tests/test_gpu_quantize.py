@@ -93,7 +93,7 @@ def test_full_size_2_30_sampled(mode):
         assert np.array_equal(got, want), s
     # properties that hold at any size, checked on the whole tensor on the device
     diff = yd.to(torch.int16) - xd.to(torch.int16)
-    assert int(diff.max()) <= 8 and int(diff.min()) >= -8    # within half a top-window LSB
+    assert int(diff.max()) <= 8 and int(diff.min()) >= -15   # half a top-window LSB up; the saturating top loses < 16
     assert bool(((xd == 0) == (yd == 0)).all())              # zeros, and only zeros, map to zero
     small = xd < 16
     assert bool((yd[small] == xd[small]).all())              # values below 16 unchanged
