@@ -57,47 +57,63 @@ SPARQ_HD uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 #endif
 }
 
+// Kernel-side copy of the placement-set constants of XformArgs.
+struct XformDev {
+    uint32_t widen_c;
+    int rounds;
+    int n;
+};
+
 // Mask of the bits BELOW the window for each of the four bytes of x (Section 3.1: the
-// window's top bit is the leading one, or the window sits at the bottom).  W = window
-// width.  widen_c / rounds move a window that landed on a disallowed placement up to
-// the next allowed one.
-template <int W>
-SPARQ_HD uint32_t drop_mask(uint32_t x, uint32_t widen_c, int rounds)
+// window's top bit is the leading one, or the window sits at the bottom).  The window
+// width is WT when WT != 0, else the run-time value w_rt.  widen_c / rounds move a
+// window that landed on a disallowed placement up to the next allowed one.
+template <int WT>
+SPARQ_HD uint32_t drop_mask(uint32_t x, int w_rt, uint32_t widen_c, int rounds)
 {
-    constexpr uint32_t LOW = 0x01010101u * (0xFFu >> W);
-    uint32_t m = (x >> W) & LOW;                 // bits of x above the lowest window
+    const int w = WT ? WT : w_rt;
+    const uint32_t low = 0x01010101u * (0xFFu >> w);
+    uint32_t m = (x >> w) & low;                 // bits of x above the lowest window
     m |= (m >> 1) & 0x7F7F7F7Fu;                 // smear the leading one downwards
-    if (8 - W > 2) m |= (m >> 2) & 0x3F3F3F3Fu;
-    if (8 - W > 4) m |= (m >> 4) & 0x0F0F0F0Fu;
+    if (!WT || 8 - WT > 2) m |= (m >> 2) & 0x3F3F3F3Fu;
+    if (!WT || 8 - WT > 4) m |= (m >> 4) & 0x0F0F0F0Fu;
     for (int r = 0; r < rounds; ++r) m |= (m << 1) & widen_c;
     return m;
 }
 
-// Trim or round four bytes given their drop masks.  Rounding adds half a window LSB;
-// a byte that would overflow 8 bits (only possible at the highest placement, where the
-// half is 0x80 >> W) keeps its trimmed value, i.e. saturates to the all-ones window.
-template <int W, bool RND>
-SPARQ_HD uint32_t apply_mask(uint32_t x, uint32_t m)
+// Trim or round four bytes given their drop masks (w = window width).  Rounding adds
+// half a window LSB; a byte that would overflow 8 bits (only possible at the highest
+// placement, where the half is 0x80 >> w) keeps its trimmed value, i.e. saturates to
+// the all-ones window.
+template <bool RND>
+SPARQ_HD uint32_t apply_mask(uint32_t x, uint32_t m, int w)
 {
     if (!RND) return x & ~m;
     uint32_t half = m ^ ((m >> 1) & 0x7F7F7F7Fu);   // (m + 1) >> 1 per byte
     uint32_t x7 = x & 0x7F7F7F7Fu, x8 = x & 0x80808080u;
     uint32_t lo = x7 + half;                        // no carry leaves a byte
     uint32_t ovf = lo & x8;                         // bit 7: x + half >= 256
-    lo -= ovf >> W;
+    lo -= ovf >> w;
     return (lo ^ x8) & ~m;
 }
 
 // T on four packed activations (bytes 0,1 and bytes 2,3 are the pairs of Eq. 2).
+// N = 2, 3, 4 fixes the window width at compile time; N = 0 takes it from d.n.
 template <int MODE, int N, bool RND>
-SPARQ_HD uint32_t xform_word(uint32_t x, uint32_t widen_c, int rounds)
+SPARQ_HD uint32_t xform_word(uint32_t x, const XformDev &d)
 {
     if (MODE == SPARQ_MODE_NONE) return x;
-    uint32_t q = apply_mask<N, RND>(x, drop_mask<N>(x, widen_c, rounds));
+    const int n = N ? N : d.n;
+    uint32_t q = apply_mask<RND>(x, drop_mask<N>(x, n, d.widen_c, d.rounds), n);
     if (MODE == SPARQ_MODE_BSPARQ) return q;
-    // vSPARQ: a byte whose partner is zero keeps the 2n-bit budget.
+    // vSPARQ: a byte whose partner is zero keeps the 2n-bit budget (all 8 bits for n = 4;
+    // a 2n-bit window at any shift 0..8-2n otherwise, Section 5.1).
     uint32_t lone = x;
-    if (2 * N < 8) lone = apply_mask<2 * N, RND>(x, drop_mask<(2 * N < 8 ? 2 * N : 4)>(x, 0u, 0));
+    if (N == 2 || N == 3) {
+        lone = apply_mask<RND>(x, drop_mask<(N == 4 ? 0 : 2 * N)>(x, 2 * n, 0u, 0), 2 * n);
+    } else if (N == 0 && 2 * n < 8) {
+        lone = apply_mask<RND>(x, drop_mask<0>(x, 2 * n, 0u, 0), 2 * n);
+    }
     uint32_t nz = ((x & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | x;   // bit 7 of each byte: byte != 0
     uint32_t partner_nz = prmt(nz, nz, 0xAB89u);           // swap within pairs, replicate bit 7
     return (q & partner_nz) | (lone & ~partner_nz);

@@ -1,10 +1,256 @@
-// placeholder until the fused kernel lands
-#include "sparq_common.cuh"
-namespace sparq { void release_gemm_state() {} }
+// Host side of the fused entry points: validation, tile-shape choice, TMA tensor maps
+// (tiled for the GEMM view, im2col for the convolution), launch.
+#include <cuda.h>
+
+#include <cstring>
+
+#include "sparq_gemm_kernel.cuh"
+
+namespace sparq {
+
+void release_gemm_state() {}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const int *, const int *, cuuint32_t, cuuint32_t,
+                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static int driver_fn(const char *name, void **fn)
+{
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPointByVersion(name, fn, 12000, cudaEnableDefault, &q);
+    if (e != cudaSuccess) return cuda_error(e, name);
+    if (q != cudaDriverEntryPointSuccess || !*fn)
+        return set_error(SPARQ_ERR_CUDA, "driver entry point %s is unavailable", name);
+    return SPARQ_OK;
+}
+
+static CUtensorMapSwizzle swizzle_for(int bk) { return bk == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B; }
+
+// 2-D K-contiguous matrix [rows][K] with row pitch ld bytes; box = bk x box_rows.
+static int encode_2d(CUtensorMap *map, const void *ptr, int64_t K, int64_t rows, int64_t ld, int bk, int box_rows)
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        int rc = driver_fn("cuTensorMapEncodeTiled", (void **)&fn);
+        if (rc != SPARQ_OK) return rc;
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld};
+    cuuint32_t box[2] = {(cuuint32_t)bk, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(bk), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return set_error(SPARQ_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return SPARQ_OK;
+}
+
+// NHWC activation tensor read as im2col columns of 128 output pixels x bk channels.
+static int encode_im2col(CUtensorMap *map, const void *ptr, int n, int h, int w, int c, int r, int s,
+                         int stride_h, int stride_w, int pad_h, int pad_w, int bk)
+{
+    static EncodeIm2colFn fn = nullptr;
+    if (!fn) {
+        int rc = driver_fn("cuTensorMapEncodeIm2col", (void **)&fn);
+        if (rc != SPARQ_OK) return rc;
+    }
+    cuuint64_t dims[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
+    cuuint64_t strides[3] = {(cuuint64_t)c, (cuuint64_t)c * w, (cuuint64_t)c * w * h};
+    // Base pixels (the filter's top-left tap) run from -pad to dim - 1 + upper.
+    int lower[2] = {-pad_w, -pad_h};
+    int upper[2] = {pad_w - (s - 1), pad_h - (r - 1)};
+    cuuint32_t estr[4] = {1, (cuuint32_t)stride_w, (cuuint32_t)stride_h, 1};
+    CUresult res = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(ptr), dims, strides, lower, upper,
+                      (cuuint32_t)bk, (cuuint32_t)kBM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(bk),
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (res != CUDA_SUCCESS) return set_error(SPARQ_ERR_CUDA, "cuTensorMapEncodeIm2col failed with CUresult %d", (int)res);
+    return SPARQ_OK;
+}
+
+static int device_info(int *sms)
+{
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_error(e, "device query");
+    if (major != 10) return set_error(SPARQ_ERR_UNSUPPORTED, "the fused kernels need an sm_100 device (found sm_%d0)", major);
+    return SPARQ_OK;
+}
+
+static int check_epilogue(const sparq_epilogue *e)
+{
+    if (!e) return set_error(SPARQ_ERR_INVALID_ARG, "sparq_epilogue is NULL");
+    if (!e->acc_out && !e->f32_out && !e->u8_out)
+        return set_error(SPARQ_ERR_INVALID_ARG, "no output requested (acc_out, f32_out and u8_out are all NULL)");
+    if ((e->f32_out || e->u8_out) && !e->scale)
+        return set_error(SPARQ_ERR_INVALID_ARG, "scale is NULL but a dequantized output is requested");
+    if ((e->acc_out && ((uintptr_t)e->acc_out & 15u)) || (e->f32_out && ((uintptr_t)e->f32_out & 15u)) ||
+        (e->u8_out && ((uintptr_t)e->u8_out & 15u)))
+        return set_error(SPARQ_ERR_UNSUPPORTED, "output pointers must be 16-byte aligned");
+    return SPARQ_OK;
+}
+
+static int pick_bn(int64_t M, int64_t N, int sms)
+{
+    const int cand[3] = {256, 128, 64};
+    const int64_t m_tiles = (M + kBM - 1) / kBM;
+    int best = 64;
+    for (int i = 0; i < 3; ++i) {
+        const int bn = cand[i];
+        if (bn > 64 && N <= bn / 2) continue;          // would be mostly padding
+        const int64_t tiles = m_tiles * ((N + bn - 1) / bn);
+        if (tiles >= sms) return bn;                    // the widest tile that still fills the GPU
+        best = bn;
+    }
+    // nothing fills the GPU: the narrowest admissible tile gives the most CTAs
+    return (N <= 64) ? 64 : best;
+}
+
+static cudaError_t launch(int bn, int bk, const CUtensorMap &ma, const CUtensorMap &mb, const GemmArgs &g,
+                          const XformArgs &x, int grid, cudaStream_t st)
+{
+    if (bn == 64 && bk == 64) return launch_gemm_shape<64, 64>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
+    if (bn == 64) return launch_gemm_shape<64, 128>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
+    if (bn == 128 && bk == 64) return launch_gemm_shape<128, 64>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
+    if (bn == 128) return launch_gemm_shape<128, 128>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
+    if (bk == 64) return launch_gemm_shape<256, 64>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
+    return launch_gemm_shape<256, 128>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
+}
+
+static void fill_common(GemmArgs *g, const XformArgs &x, const sparq_epilogue *e, unsigned int *status)
+{
+    g->xf = XformDev{x.widen_c, x.widen_rounds, x.n};
+    g->scale = e->scale;
+    g->bias = e->bias;
+    g->relu = e->relu ? 1 : 0;
+    g->inv_out_scale = e->inv_out_scale;
+    g->acc_out = e->acc_out;
+    g->f32_out = e->f32_out;
+    g->u8_out = e->u8_out;
+    g->status = status;
+}
+
+static int gemm_impl(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb, int64_t M, int64_t N, int64_t K,
+                     const XformArgs &x, const sparq_epilogue *e, cudaStream_t st)
+{
+    int sms = 0;
+    int rc = device_info(&sms);
+    if (rc != SPARQ_OK) return rc;
+    unsigned int *status = nullptr;
+    rc = get_status_word(&status);
+    if (rc != SPARQ_OK) return rc;
+
+    // reduction step: the one that pads K the least; ties go to the wider step
+    const int64_t pad128 = (K + 127) / 128 * 128, pad64 = (K + 63) / 64 * 64;
+    const int bk = (pad64 < pad128) ? 64 : 128;
+    const int bn = pick_bn(M, N, sms);
+
+    CUtensorMap ma, mb;
+    rc = encode_2d(&ma, A, K, M, lda, bk, kBM);
+    if (rc != SPARQ_OK) return rc;
+    rc = encode_2d(&mb, B, K, N, ldb, bk, bn);
+    if (rc != SPARQ_OK) return rc;
+
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.M = M; g.N = N; g.K = K;
+    g.k_blocks = (int)((K + bk - 1) / bk);
+    fill_common(&g, x, e, status);
+    const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
+    if (ce != cudaSuccess) return cuda_error(ce, "sparq_gemm_kernel launch");
+    return SPARQ_OK;
+}
+
+}  // namespace sparq
+
 using namespace sparq;
-extern "C" int sparq_gemm_s8(const uint8_t *, int64_t, const int8_t *, int64_t, int64_t, int64_t, int64_t,
-                             const sparq_params *, const sparq_epilogue *, void *)
-{ return set_error(SPARQ_ERR_UNSUPPORTED, "not built yet"); }
-extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *, int, int, int, int, const int8_t *, int, int, int,
-                                    int, int, int, int, const sparq_params *, const sparq_epilogue *, void *)
-{ return set_error(SPARQ_ERR_UNSUPPORTED, "not built yet"); }
+
+extern "C" int sparq_gemm_s8(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                             int64_t M, int64_t N, int64_t K,
+                             const sparq_params *p, const sparq_epilogue *e, void *stream)
+{
+    XformArgs x;
+    int rc = validate_params(p, &x);
+    if (rc != SPARQ_OK) return rc;
+    rc = check_epilogue(e);
+    if (rc != SPARQ_OK) return rc;
+    if (M < 0 || N < 0 || K < 0) return set_error(SPARQ_ERR_INVALID_ARG, "negative dimension");
+    if (M == 0 || N == 0) return SPARQ_OK;
+    if (!A || !B) return set_error(SPARQ_ERR_INVALID_ARG, "A or B is NULL");
+    if (K == 0 || K % 16 || K > 65536) return set_error(SPARQ_ERR_UNSUPPORTED, "K = %lld must be a multiple of 16 in [16, 65536]", (long long)K);
+    if (lda < K || ldb < K || lda % 16 || ldb % 16)
+        return set_error(SPARQ_ERR_UNSUPPORTED, "lda/ldb must be multiples of 16 and at least K");
+    if (((uintptr_t)A | (uintptr_t)B) & 15u) return set_error(SPARQ_ERR_UNSUPPORTED, "A and B must be 16-byte aligned");
+    if (M > (int64_t)1 << 31 || N > (int64_t)1 << 31) return set_error(SPARQ_ERR_UNSUPPORTED, "M or N too large");
+    return gemm_impl(A, lda, B, ldb, M, N, K, x, e, (cudaStream_t)stream);
+}
+
+extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, int c,
+                                    const int8_t *wgt, int cout, int r, int s,
+                                    int stride_h, int stride_w, int pad_h, int pad_w,
+                                    const sparq_params *p, const sparq_epilogue *e, void *stream)
+{
+    XformArgs x;
+    int rc = validate_params(p, &x);
+    if (rc != SPARQ_OK) return rc;
+    rc = check_epilogue(e);
+    if (rc != SPARQ_OK) return rc;
+    if (n < 0 || h < 0 || w < 0 || c < 0 || cout < 0) return set_error(SPARQ_ERR_INVALID_ARG, "negative dimension");
+    if (r < 1 || s < 1 || stride_h < 1 || stride_w < 1 || pad_h < 0 || pad_w < 0)
+        return set_error(SPARQ_ERR_INVALID_ARG, "filter size and strides must be >= 1, pads >= 0");
+    if (r > 7 || s > 7 || stride_h > 8 || stride_w > 8 || pad_h >= r || pad_w >= s)
+        return set_error(SPARQ_ERR_UNSUPPORTED, "filter up to 7x7, strides up to 8, pads below the filter size");
+    if (n == 0 || cout == 0) return SPARQ_OK;
+    if (h + 2 * pad_h < r || w + 2 * pad_w < s) return set_error(SPARQ_ERR_INVALID_ARG, "filter larger than the padded image");
+    if (!x_in || !wgt) return set_error(SPARQ_ERR_INVALID_ARG, "x or wgt is NULL");
+    if (c == 0 || c % 16) return set_error(SPARQ_ERR_UNSUPPORTED, "c = %d must be a positive multiple of 16", c);
+    if (((uintptr_t)x_in | (uintptr_t)wgt) & 15u) return set_error(SPARQ_ERR_UNSUPPORTED, "x and wgt must be 16-byte aligned");
+    const int ho = (h + 2 * pad_h - r) / stride_h + 1;
+    const int wo = (w + 2 * pad_w - s) / stride_w + 1;
+    const int64_t M = (int64_t)n * ho * wo;
+    const int64_t K = (int64_t)r * s * c;
+    if (K > 65536) return set_error(SPARQ_ERR_UNSUPPORTED, "r*s*c = %lld exceeds 65536", (long long)K);
+    cudaStream_t st = (cudaStream_t)stream;
+
+    // A 1x1 filter with unit stride reads the NHWC tensor as the M x c matrix it already is.
+    if (r == 1 && s == 1 && stride_h == 1 && stride_w == 1 && pad_h == 0 && pad_w == 0)
+        return gemm_impl(x_in, c, wgt, c, M, cout, c, x, e, st);
+
+    if (c % 64) return set_error(SPARQ_ERR_UNSUPPORTED, "c = %d must be a multiple of 64 for filters other than 1x1 stride 1", c);
+    int sms = 0;
+    rc = device_info(&sms);
+    if (rc != SPARQ_OK) return rc;
+    unsigned int *status = nullptr;
+    rc = get_status_word(&status);
+    if (rc != SPARQ_OK) return rc;
+    const int bk = (c % 128 == 0) ? 128 : 64;
+    const int bn = pick_bn(M, cout, sms);
+    CUtensorMap ma, mb;
+    rc = encode_im2col(&ma, x_in, n, h, w, c, r, s, stride_h, stride_w, pad_h, pad_w, bk);
+    if (rc != SPARQ_OK) return rc;
+    rc = encode_2d(&mb, wgt, K, cout, K, bk, bn);
+    if (rc != SPARQ_OK) return rc;
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.M = M; g.N = cout; g.K = K;
+    g.k_blocks = (int)(K / bk);
+    g.conv = 1;
+    g.c_blocks = c / bk;
+    g.S = s;
+    g.Ho = ho; g.Wo = wo;
+    g.stride_h = stride_h; g.stride_w = stride_w; g.pad_h = pad_h; g.pad_w = pad_w;
+    fill_common(&g, x, e, status);
+    const int64_t tiles = ((M + kBM - 1) / kBM) * ((cout + bn - 1) / bn);
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
+    if (ce != cudaSuccess) return cuda_error(ce, "sparq_gemm_kernel (convolution) launch");
+    return SPARQ_OK;
+}

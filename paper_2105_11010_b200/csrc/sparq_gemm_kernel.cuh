@@ -1,0 +1,506 @@
+// Fused SPARQ GEMM / implicit-GEMM convolution for sm_100a.
+//
+//   acc[m][j] = sum_k T(A)[m][k] * B[j][k]      (Eq. 1 with Eq. 2 applied on the fly)
+//
+// One persistent CTA per SM walks output tiles of 128 x BN.  Warp roles:
+//   warp 0        TMA producer: A tile (tiled 2-D box for the GEMM, im2col box for the
+//                 convolution) and B tile into a ring of shared-memory stages
+//   warp 1        allocates tensor memory; one lane issues tcgen05.mma kind::i8
+//                 (u8 x s8 -> s32) on each transformed stage
+//   warps 2..5    epilogue: tcgen05.ld of a finished accumulator, fp32 scale / bias /
+//                 ReLU / requantize, global stores
+//   warps 6..13   transform: rewrite the A stage in place with bSPARQ / vSPARQ
+//
+// A stage travels  TMA (async proxy) -> transform warps (generic proxy) -> MMA (async
+// proxy); the hand-offs are mbarriers, with fence.proxy.async after the in-place rewrite.
+// The 128-byte (64-byte) shared-memory swizzle only permutes 16-byte chunks inside a
+// row, and a vSPARQ pair never straddles a 16-byte chunk, so the transform treats the
+// stage as a flat array of 16-byte vectors.
+//
+// Every wait is bounded: when a wait gives up it sets bit 0 of the status word, raises a
+// CTA-wide abort flag that makes all later waits return at once, and the kernel still
+// runs to its normal end (loops have fixed trip counts), drains its own copies and frees
+// its tensor memory.
+#pragma once
+
+#include <cuda.h>
+
+#include "sparq_common.cuh"
+
+namespace sparq {
+
+constexpr int kBM = 128;                 // rows of an output tile = MMA M
+constexpr int kNumEpiWarps = 4;
+constexpr int kNumXfWarps = 8;
+constexpr int kFirstEpiWarp = 2;
+constexpr int kFirstXfWarp = kFirstEpiWarp + kNumEpiWarps;
+constexpr int kGemmThreads = 32 * (kFirstXfWarp + kNumXfWarps);
+constexpr int kSmemBudget = 200 * 1024;  // for the stage ring
+constexpr long long kWaitLimitCycles = 2000000000LL;
+
+struct GemmArgs {
+    // problem
+    int64_t M, N, K;        // GEMM view (K = r*s*c for the convolution)
+    int k_blocks;           // number of BK-wide reduction steps
+    // convolution geometry (conv = 1) for the im2col producer
+    int conv;
+    int c_blocks;           // BK-wide channel blocks per filter tap
+    int S;                  // filter width (taps are ordered r-major, s-minor)
+    int Ho, Wo;
+    int stride_h, stride_w, pad_h, pad_w;
+    // transform
+    XformDev xf;
+    // epilogue
+    const float *scale;
+    const float *bias;
+    int relu;
+    float inv_out_scale;
+    int32_t *acc_out;
+    float *f32_out;
+    uint8_t *u8_out;
+    unsigned int *status;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false (after flagging) if the phase did not complete in time or
+// if another thread of the CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          unsigned int *status, bool ignore_abort = false)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    if (!ignore_abort && *abort_flag) return false;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 0x3FFu) == 0) {
+            if (!ignore_abort && *abort_flag) return false;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                *abort_flag = 1u;
+                atomicOr(status, 1u);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+// im2col box: `pixels-per-column` output pixels starting at base pixel (w, h, n), channels
+// c .. c+box, filter tap offset (woff, hoff); out-of-image taps are filled with zeros.
+__device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                                   int c, int w, int h, int n, uint16_t woff, uint16_t hoff)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        :: "r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(woff), "h"(hoff) : "memory");
+}
+
+__device__ __forceinline__ void fence_proxy_async_smem()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem], 128 x N x 32, u8 x s8 -> s32.
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are ROW_BYTES long
+// (128 or 64) and swizzled with the matching TMA mode; 8-row groups are contiguous.
+template <int ROW_BYTES>
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
+{
+    constexpr uint64_t layout = (ROW_BYTES == 128) ? 2ull : 4ull;   // 128B / 64B swizzle
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);            // start address
+    d |= (uint64_t)1 << 16;                              // leading-dimension offset (unused when swizzled)
+    d |= (uint64_t)((8 * ROW_BYTES) >> 4) << 32;         // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                              // descriptor version of this architecture
+    d |= layout << 61;
+    return d;
+}
+
+// kind::i8 instruction descriptor: s32 accumulator, unsigned A, signed B, both K-major.
+__device__ __forceinline__ constexpr uint32_t make_idesc_i8(int n)
+{
+    return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
+
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ---- epilogue arithmetic ----------------------------------------------------------------
+
+// int32 accumulator -> (fp32 value, requantized byte), one IEEE operation per step.
+__device__ __forceinline__ float dequant(int32_t acc, float scale, float bias, int relu)
+{
+    float t = __int2float_rn(acc);
+    float y = __fmaf_rn(t, scale, bias);
+    if (relu) y = (y > 0.0f) ? y : 0.0f;
+    return y;
+}
+
+__device__ __forceinline__ uint32_t requant(float y, float inv_out_scale)
+{
+    float u = rintf(__fmul_rn(y, inv_out_scale));
+    if (!(u > 0.0f)) return 0u;          // negative, zero and NaN
+    if (u > 255.0f) return 255u;
+    return (uint32_t)u;
+}
+
+// ---- the kernel ---------------------------------------------------------------------------
+
+template <int BN, int BK>
+struct TileCfg {
+    static constexpr int kABytes = kBM * BK;
+    static constexpr int kBBytes = BN * BK;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kStagesRaw = kSmemBudget / kStageBytes;
+    static constexpr int kStages = kStagesRaw > 8 ? 8 : kStagesRaw;
+    static constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;   // two accumulators
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024; // + alignment slack
+};
+
+template <int BN, int BK, int MODE, int XN, bool RND>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const GemmArgs g)
+{
+    using Cfg = TileCfg<BN, BK>;
+    constexpr int S = Cfg::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[S], bar_xf[S], bar_empty[S];
+    __shared__ __align__(8) uint64_t bar_acc_full[2], bar_acc_empty[2], bar_done;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ uint32_t abort_word;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    volatile uint32_t *abort_flag = &abort_word;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    auto a_stage = [&](int s) { return smem_base + (uint32_t)s * Cfg::kStageBytes; };
+    auto b_stage = [&](int s) { return smem_base + (uint32_t)s * Cfg::kStageBytes + Cfg::kABytes; };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_xf[s]), kNumXfWarps);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&bar_acc_full[a]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[a]), kNumEpiWarps);
+        }
+        mbar_init(smem_u32(&bar_done), 1);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     :: "r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)Cfg::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    const int64_t m_tiles = (g.M + kBM - 1) / kBM;
+    const int64_t n_tiles = (g.N + BN - 1) / BN;
+    const int64_t total_tiles = m_tiles * n_tiles;
+    const int kb_count = g.k_blocks;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            uint32_t it = 0;   // running stage counter across tiles
+            for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+                const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
+                const int64_t m0 = mt * kBM;
+                const int n0 = (int)(nt * BN);
+                int base_w = 0, base_h = 0, base_n = 0;
+                if (g.conv) {
+                    const int64_t hw = (int64_t)g.Ho * g.Wo;
+                    base_n = (int)(m0 / hw);
+                    const int rem = (int)(m0 % hw);
+                    base_h = (rem / g.Wo) * g.stride_h - g.pad_h;
+                    base_w = (rem % g.Wo) * g.stride_w - g.pad_w;
+                }
+                for (int kb = 0; kb < kb_count; ++kb, ++it) {
+                    const int s = it % S;
+                    const uint32_t use = it / S;
+                    if (use > 0) mbar_wait(smem_u32(&bar_empty[s]), (use - 1) & 1, abort_flag, g.status);
+                    if (*abort_flag) break;   // stop issuing copies once the CTA has given up
+                    const uint32_t full = smem_u32(&bar_full[s]);
+                    mbar_expect_tx(full, Cfg::kStageBytes);
+                    if (g.conv) {
+                        const int tap = kb / g.c_blocks, cb = kb % g.c_blocks;
+                        tma_load_im2col_4d(a_stage(s), &map_a, full, cb * BK, base_w, base_h, base_n,
+                                           (uint16_t)(tap % g.S), (uint16_t)(tap / g.S));
+                    } else {
+                        tma_load_2d(a_stage(s), &map_a, full, kb * BK, (int)m0);
+                    }
+                    tma_load_2d(b_stage(s), &map_b, full, kb * BK, n0);
+                }
+                if (*abort_flag) break;
+            }
+            // After an abort: wait (bounded) for the copies this thread still has in
+            // flight, so that none lands after the CTA has exited.
+            if (*abort_flag) {
+                const uint32_t first = it > (uint32_t)S ? it - S : 0;
+                for (uint32_t j = first; j < it; ++j)
+                    mbar_wait(smem_u32(&bar_full[j % S]), (j / S) & 1, abort_flag, g.status, true);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_i8(BN);
+            uint32_t it = 0, local_tile = 0;
+            for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
+                const int acc = local_tile & 1;
+                const uint32_t acc_use = local_tile >> 1;
+                if (acc_use > 0) mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status);
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < kb_count; ++kb, ++it) {
+                    const int s = it % S;
+                    const uint32_t ph = (it / S) & 1;
+                    if (MODE == SPARQ_MODE_NONE) mbar_wait(smem_u32(&bar_full[s]), ph, abort_flag, g.status);
+                    else mbar_wait(smem_u32(&bar_xf[s]), ph, abort_flag, g.status);
+                    tc_fence_after();
+                    const uint64_t adesc = make_smem_desc<BK>(a_stage(s));
+                    const uint64_t bdesc = make_smem_desc<BK>(b_stage(s));
+#pragma unroll
+                    for (int k = 0; k < BK / 32; ++k)
+                        tc_mma_i8(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
+                                  (kb > 0 || k > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&bar_empty[s]));       // stage reusable once these MMAs retire
+                }
+                tc_commit(smem_u32(&bar_acc_full[acc]));      // accumulator complete
+            }
+            // all tensor-core work of this CTA has retired before tensor memory is freed
+            tc_commit(smem_u32(&bar_done));
+            mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, true);
+        }
+        __syncwarp();
+    } else if (warp < kFirstXfWarp) {
+        // ================= epilogue =================
+        const int quarter = warp & 3;                   // tensor-memory lanes this warp may read
+        uint32_t local_tile = 0;
+        const bool vec_ok = (g.N % 16) == 0;
+        for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
+            const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
+            const int acc = local_tile & 1;
+            const uint32_t acc_use = local_tile >> 1;
+            mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status);
+            tc_fence_after();
+            const int64_t row = mt * kBM + quarter * 32 + lane;
+            const bool row_ok = row < g.M;
+#pragma unroll 1
+            for (int ch = 0; ch < BN / 32; ++ch) {
+                uint32_t r[32];
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + ch * 32);
+                tmem_ld_32x32(taddr, r);
+                const int64_t col0 = nt * BN + ch * 32;
+                if (!row_ok || col0 >= g.N) continue;
+                const int64_t off = row * g.N + col0;
+                const bool full = vec_ok && (col0 + 32 <= g.N);
+                if (g.acc_out) {
+                    if (full) {
+                        int4 *dst = reinterpret_cast<int4 *>(g.acc_out + off);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            dst[v] = make_int4((int)r[4 * v], (int)r[4 * v + 1], (int)r[4 * v + 2], (int)r[4 * v + 3]);
+                    } else {
+                        for (int i = 0; i < 32 && col0 + i < g.N; ++i) g.acc_out[off + i] = (int32_t)r[i];
+                    }
+                }
+                if (g.f32_out || g.u8_out) {
+                    float y[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int64_t c = col0 + i;
+                        const bool ok = c < g.N;
+                        const float sc = ok ? __ldg(g.scale + c) : 0.0f;
+                        const float bi = (ok && g.bias) ? __ldg(g.bias + c) : 0.0f;
+                        y[i] = dequant((int32_t)r[i], sc, bi, g.relu);
+                    }
+                    if (g.f32_out) {
+                        if (full) {
+                            float4 *dst = reinterpret_cast<float4 *>(g.f32_out + off);
+#pragma unroll
+                            for (int v = 0; v < 8; ++v) dst[v] = make_float4(y[4 * v], y[4 * v + 1], y[4 * v + 2], y[4 * v + 3]);
+                        } else {
+                            for (int i = 0; i < 32 && col0 + i < g.N; ++i) g.f32_out[off + i] = y[i];
+                        }
+                    }
+                    if (g.u8_out) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            w[v] = requant(y[4 * v], g.inv_out_scale) | (requant(y[4 * v + 1], g.inv_out_scale) << 8) |
+                                   (requant(y[4 * v + 2], g.inv_out_scale) << 16) | (requant(y[4 * v + 3], g.inv_out_scale) << 24);
+                        if (full) {
+                            uint4 *dst = reinterpret_cast<uint4 *>(g.u8_out + off);
+                            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                        } else {
+                            for (int i = 0; i < 32 && col0 + i < g.N; ++i)
+                                g.u8_out[off + i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
+        }
+    } else if (MODE != SPARQ_MODE_NONE) {
+        // ================= transform =================
+        const int xt = threadIdx.x - kFirstXfWarp * 32;            // 0 .. 255
+        constexpr int kXfThreads = kNumXfWarps * 32;
+        constexpr int kVecs = Cfg::kABytes / 16;
+        constexpr int kPerThread = kVecs / kXfThreads;
+        static_assert(kVecs % kXfThreads == 0, "A stage must split evenly over the transform threads");
+        const XformDev xf = g.xf;
+        uint32_t it = 0;
+        for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            for (int kb = 0; kb < kb_count; ++kb, ++it) {
+                const int s = it % S;
+                mbar_wait(smem_u32(&bar_full[s]), (it / S) & 1, abort_flag, g.status);
+                const uint32_t base = a_stage(s) + (uint32_t)xt * 16u;
+                uint4 v[kPerThread];
+#pragma unroll
+                for (int j = 0; j < kPerThread; ++j)
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w)
+                                 : "r"(base + (uint32_t)(j * kXfThreads * 16)));
+#pragma unroll
+                for (int j = 0; j < kPerThread; ++j) {
+                    v[j].x = xform_word<MODE, XN, RND>(v[j].x, xf);
+                    v[j].y = xform_word<MODE, XN, RND>(v[j].y, xf);
+                    v[j].z = xform_word<MODE, XN, RND>(v[j].z, xf);
+                    v[j].w = xform_word<MODE, XN, RND>(v[j].w, xf);
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
+                                 :: "r"(base + (uint32_t)(j * kXfThreads * 16)),
+                                    "r"(v[j].x), "r"(v[j].y), "r"(v[j].z), "r"(v[j].w) : "memory");
+                }
+                fence_proxy_async_smem();       // generic-proxy writes visible to the tensor core
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_xf[s]));
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     :: "r"(tmem_base), "r"((uint32_t)Cfg::kTmemCols) : "memory");
+    }
+}
+
+// Host launcher for one tile shape; picks the transform variant.  Defined once per
+// (BN, BK) in its own translation unit.
+template <int BN, int BK>
+cudaError_t launch_gemm_shape(const CUtensorMap &ma, const CUtensorMap &mb, const GemmArgs &g,
+                              int mode, int n, int rnd, int grid, cudaStream_t st);
+
+#define SPARQ_LAUNCH_VARIANT(MODE_, XN_, RND_)                                                         \
+    do {                                                                                               \
+        auto kfn = sparq_gemm_kernel<BN, BK, MODE_, XN_, RND_>;                                        \
+        cudaError_t e_ = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
+                                              TileCfg<BN, BK>::kSmemBytes);                            \
+        if (e_ != cudaSuccess) return e_;                                                              \
+        kfn<<<grid, kGemmThreads, TileCfg<BN, BK>::kSmemBytes, st>>>(ma, mb, g);                       \
+        return cudaGetLastError();                                                                     \
+    } while (0)
+
+#define SPARQ_DEFINE_GEMM_SHAPE(BN_, BK_)                                                              \
+    template <>                                                                                        \
+    cudaError_t launch_gemm_shape<BN_, BK_>(const CUtensorMap &ma, const CUtensorMap &mb,              \
+                                            const GemmArgs &g, int mode, int n, int rnd, int grid,     \
+                                            cudaStream_t st)                                           \
+    {                                                                                                  \
+        constexpr int BN = BN_, BK = BK_;                                                              \
+        if (mode == SPARQ_MODE_NONE) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_NONE, 4, false);                  \
+        if (mode == SPARQ_MODE_BSPARQ) {                                                               \
+            if (n == 4) { if (rnd) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_BSPARQ, 4, true);                   \
+                          else SPARQ_LAUNCH_VARIANT(SPARQ_MODE_BSPARQ, 4, false); }                    \
+            if (rnd) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_BSPARQ, 0, true);                                 \
+            else SPARQ_LAUNCH_VARIANT(SPARQ_MODE_BSPARQ, 0, false);                                    \
+        }                                                                                              \
+        if (n == 4) { if (rnd) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_VSPARQ, 4, true);                       \
+                      else SPARQ_LAUNCH_VARIANT(SPARQ_MODE_VSPARQ, 4, false); }                        \
+        if (rnd) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_VSPARQ, 0, true);                                     \
+        else SPARQ_LAUNCH_VARIANT(SPARQ_MODE_VSPARQ, 0, false);                                        \
+    }
+
+}  // namespace sparq

@@ -31,8 +31,7 @@ __device__ __forceinline__ void st_stream(uint4 *p, uint4 v)
 
 template <int MODE, int N, bool RND>
 __global__ void __launch_bounds__(kThreads)
-quantize_vec_kernel(const uint4 *in, uint4 *out, size_t nvec,
-                    uint32_t widen_c, int rounds)
+quantize_vec_kernel(const uint4 *in, uint4 *out, size_t nvec, XformDev d)
 {
     const size_t tile = (size_t)kThreads * kVec;
     for (size_t base = (size_t)blockIdx.x * tile; base < nvec; base += (size_t)gridDim.x * tile) {
@@ -47,10 +46,10 @@ quantize_vec_kernel(const uint4 *in, uint4 *out, size_t nvec,
         for (int j = 0; j < kVec; ++j) {
             if (idx[j] < nvec) {
                 uint4 o;
-                o.x = xform_word<MODE, N, RND>(v[j].x, widen_c, rounds);
-                o.y = xform_word<MODE, N, RND>(v[j].y, widen_c, rounds);
-                o.z = xform_word<MODE, N, RND>(v[j].z, widen_c, rounds);
-                o.w = xform_word<MODE, N, RND>(v[j].w, widen_c, rounds);
+                o.x = xform_word<MODE, N, RND>(v[j].x, d);
+                o.y = xform_word<MODE, N, RND>(v[j].y, d);
+                o.z = xform_word<MODE, N, RND>(v[j].z, d);
+                o.w = xform_word<MODE, N, RND>(v[j].w, d);
                 st_stream(out + idx[j], o);
             }
         }
@@ -108,10 +107,11 @@ template <int MODE, int N>
 static cudaError_t launch_vec(const uint4 *in, uint4 *out, size_t nvec, const XformArgs &a,
                               int blocks, cudaStream_t st)
 {
+    XformDev d{a.widen_c, a.widen_rounds, a.n};
     if (a.rnd)
-        quantize_vec_kernel<MODE, N, true><<<blocks, kThreads, 0, st>>>(in, out, nvec, a.widen_c, a.widen_rounds);
+        quantize_vec_kernel<MODE, N, true><<<blocks, kThreads, 0, st>>>(in, out, nvec, d);
     else
-        quantize_vec_kernel<MODE, N, false><<<blocks, kThreads, 0, st>>>(in, out, nvec, a.widen_c, a.widen_rounds);
+        quantize_vec_kernel<MODE, N, false><<<blocks, kThreads, 0, st>>>(in, out, nvec, d);
     return cudaGetLastError();
 }
 
