@@ -21,4 +21,5 @@ from .generators import (  # noqa: F401
     ConvShape,
     resnet50_conv_layers,
     conv_out_hw,
+    inv_out_scale,
 )

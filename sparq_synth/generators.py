@@ -127,3 +127,14 @@ def resnet50_conv_layers() -> List[ConvShape]:
             index[key] = len(merged)
             merged.append(c)
     return merged
+
+
+def inv_out_scale(k: int, zero_frac: float = 0.5) -> float:
+    """A fixed requantization multiplier for a layer with reduction length ``k``.
+
+    With the value recipe above an accumulator has a standard deviation of about
+    ``sqrt(k * (1 - zero_frac) * 1600 * 900)`` and the mean per-channel scale is
+    0.0055; the multiplier maps one standard deviation of the dequantized output
+    to 40 on the next layer's uint8 grid (the activations' own half-normal)."""
+    sigma_acc = (k * (1.0 - zero_frac) * 1600.0 * 900.0) ** 0.5
+    return float(np.float32(40.0 / (sigma_acc * 0.0055)))
