@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the SPARQ hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras]
+
+A step is one pass of the whole hot path -- vSPARQ transform (n = 4, five placements,
+round to nearest), u8 x s8 -> s32 implicit-GEMM convolution, fp32 scale + bias + ReLU +
+requantize to uint8 -- over one batch of the ResNet-18-style workload
+(32 x 56 x 56 x 64 NHWC uint8 activations with 45 % zeros, 64 filters of 3x3, stride 1,
+pad 1).  One fused kernel launch per step.  Prints one JSON line.
+
+With --impl reference the CPU oracle is timed instead (rank 0 only): each step is the
+same layer on a bounded number of images.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import sparq_synth as synth  # noqa: E402
+
+METRIC = "fused SPARQ INT8 conv TOPS"
+UNIT = "TOPS"
+
+# ResNet-18-style layer the metric is quoted on
+NB, H, W, C, COUT, R, S, STRIDE, PAD = 32, 56, 56, 64, 64, 3, 3, 1, 1
+ZERO_FRAC = 0.45
+SEED = 1
+OPS_PER_STEP = 2 * NB * H * W * COUT * R * S * C          # dense count: no MAC is skipped
+IN_BYTES = NB * H * W * C
+OUT_BYTES = NB * H * W * COUT
+WGT_BYTES = COUT * R * S * C
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
+INT8_OVER_BF16 = 2.0     # nominal dense ratio (4.5 POPS int8 vs 2.25 PFLOPS bf16)
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=FALLBACK_HBM_GBS, bf16=FALLBACK_BF16_TFLOPS, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.gpu_index)],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [t.strip() for t in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def build_layer(device, sets):
+    """`sets` independent input / output buffer pairs (rotated so that consecutive steps
+    never find their operands in L2) and the resident layer parameters."""
+    import torch
+    xs = [torch.from_numpy(synth.activations(SEED, (NB, H, W, C), ZERO_FRAC, stream=10 + i)).to(device)
+          for i in range(sets)]
+    outs = [torch.empty((NB, H, W, COUT), dtype=torch.uint8, device=device) for _ in range(sets)]
+    wt = torch.from_numpy(synth.weights(SEED, (COUT, R, S, C))).to(device)
+    scale = torch.from_numpy(synth.scales(SEED, COUT)).to(device)
+    bias = torch.from_numpy(synth.bias(SEED, COUT)).to(device)
+    return xs, outs, wt, scale, bias
+
+
+def time_region(fn, steps, warmup, sync):
+    import torch
+    for i in range(warmup):
+        fn(i)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync()
+    e0.record()
+    for i in range(steps):
+        fn(warmup + i)
+    e1.record()
+    sync()
+    return e0.elapsed_time(e1)      # ms
+
+
+def extras(device, pk, steps):
+    """Other workloads of the same library, each with its own roofline: the standalone
+    transform on 2^30 activations and the ResNet-50 layer sweep at batch 64."""
+    import torch
+    import paper_2105_11010_b200 as sparq
+    out = {}
+    sync = torch.cuda.synchronize
+    # --- standalone transform: 2^30 uint8 in, 2^30 out, 50 % zeros ---
+    n = 1 << 30
+    gen = torch.Generator(device=device).manual_seed(4)
+    x = torch.empty(n, dtype=torch.uint8, device=device)
+    chunk = 1 << 26
+    for lo in range(0, n, chunk):
+        z = torch.randn(chunk, generator=gen, device=device)
+        v = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
+        v[torch.rand(chunk, generator=gen, device=device) < 0.5] = 0
+        x[lo:lo + chunk] = v
+    y = torch.empty_like(x)
+    tr = {}
+    for name, mode in (("bsparq", sparq.MODE_BSPARQ), ("vsparq", sparq.MODE_VSPARQ)):
+        p = sparq.SparqParams(mode, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+        ms = time_region(lambda i: sparq.sparq_quantize(x, y, 1 << 20, 1024, p), 20, 3, sync) / 20
+        gbs = 2 * n / ms / 1e6
+        tr[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1),
+                    "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
+                                 "frac": round(gbs / pk["hbm"], 4), "traffic": None,
+                                 "peak_source": pk["source"] + " copy"}}
+    out["transform_2p30"] = tr
+    del x, y
+    # --- ResNet-50 sweep, batch 64, every conv shape (22 shapes, 52 instances) ---
+    p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+    layers, total_ms, total_ops = [], 0.0, 0
+    for li, L in enumerate(synth.resnet50_conv_layers()):
+        zf = float(np.random.default_rng(100 + li).uniform(0.3, 0.7))
+        ho, wo = L.out_hw()
+        in_b = 64 * L.h * L.w * L.cin
+        sets = max(2, min(8, int(1.2 * L2_BYTES // (in_b + 64 * ho * wo * L.cout)) + 1))
+        g = torch.Generator(device=device).manual_seed(100 + li)
+        xs = []
+        for _ in range(sets):
+            z = torch.randn(in_b, generator=g, device=device)
+            v = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
+            v[torch.rand(in_b, generator=g, device=device) < zf] = 0
+            xs.append(v.view(64, L.h, L.w, L.cin))
+        os_ = [torch.empty((64, ho, wo, L.cout), dtype=torch.uint8, device=device) for _ in range(sets)]
+        wt = torch.from_numpy(synth.weights(100 + li, (L.cout, L.r, L.s, L.cin))).to(device)
+        sc = torch.from_numpy(synth.scales(100 + li, L.cout)).to(device)
+        bi = torch.from_numpy(synth.bias(100 + li, L.cout)).to(device)
+        inv = synth.inv_out_scale(L.r * L.s * L.cin, zf)
+
+        def step(i, xs=xs, os_=os_, wt=wt, sc=sc, bi=bi, inv=inv, L=L):
+            sparq.sparq_conv2d_nhwc_s8(xs[i % len(xs)], wt, (L.stride, L.stride), (L.pad, L.pad), p,
+                                       scale=sc, bias=bi, relu=True, inv_out_scale=inv, u8_out=os_[i % len(xs)])
+        ms = time_region(step, steps, 3, sync) / steps
+        ops = L.ops(64)
+        layers.append({"layer": f"{L.h}x{L.w}x{L.cin}->{L.cout} {L.r}x{L.s}/s{L.stride}", "count": L.count,
+                       "ms": round(ms, 4), "tops": round(ops / ms / 1e9, 1)})
+        total_ms += ms * L.count
+        total_ops += ops * L.count
+        del xs, os_
+    sparq.sparq_check()
+    tops = total_ops / total_ms / 1e9
+    int8_peak = pk["bf16"] * INT8_OVER_BF16
+    out["resnet50_sweep_b64"] = {"ms_per_pass": round(total_ms, 3), "tops": round(tops, 1),
+                                 "frac_of_int8_peak": round(tops / int8_peak, 4), "layers": layers}
+    return out
+
+
+def cpu_baseline(images: int):
+    """The oracle as it stands on the host cores, on `images` images of the same layer."""
+    import oracle
+    x = synth.activations(SEED, (images, H, W, C), ZERO_FRAC, stream=10)
+    wt = synth.weights(SEED, (COUT, R, S, C))
+    scale, bias = synth.scales(SEED, COUT), synth.bias(SEED, COUT)
+    inv = synth.inv_out_scale(R * S * C, ZERO_FRAC)
+    t0 = time.perf_counter()
+    acc = oracle.conv2d_nhwc(x, wt, (STRIDE, STRIDE), (PAD, PAD), oracle.MODE_VSPARQ, 4, 0x1F, 1)
+    oracle.epilogue(acc, scale, bias, True, inv)
+    dt = time.perf_counter() - t0
+    ops = 2 * images * H * W * COUT * R * S * C
+    return ops / dt / 1e12, dt, oracle.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    images = 2
+    for _ in range(args.warmup):
+        cpu_baseline(images)
+    t0 = time.perf_counter()
+    cores = 1
+    for _ in range(args.steps):
+        _, _, cores = cpu_baseline(images)
+    dt = time.perf_counter() - t0
+    value = args.steps * 2 * images * H * W * COUT * R * S * C / dt / 1e12
+    sample = f"{images} of {NB} images per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": "resnet18_conv3x3_b32_56x56x64_to_64 (CPU oracle, " + sample + ")"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the transform and ResNet-50 sweep sections")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        if args.steps == 400:
+            args.steps = 20
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2105_11010_b200 as sparq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the SPARQ library has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def sync():
+        torch.cuda.synchronize()
+
+    pk = peaks()
+    sets = 20   # 20 x (6.4 MB in + 6.4 MB out) = 257 MB > 126 MB of L2
+    xs, outs, wt, scale, bias = build_layer(device, sets)
+    inv = synth.inv_out_scale(R * S * C, ZERO_FRAC)
+    params = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+
+    def step(i):
+        j = i % sets
+        sparq.sparq_conv2d_nhwc_s8(xs[j], wt, (STRIDE, STRIDE), (PAD, PAD), params, scale=scale, bias=bias,
+                                   relu=True, inv_out_scale=inv, u8_out=outs[j])
+
+    for i in range(args.warmup):
+        step(i)
+    sampler = ClockSampler(local)
+    sync(); barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync(); barrier()
+    e0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    e1.record()
+    sync(); barrier()
+    ms_total = e0.elapsed_time(e1)
+    # keep the GPU busy a little longer so that the clock sampler sees it under load
+    t_end = time.time() + 0.6
+    i = 0
+    while time.time() < t_end:
+        step(i); i += 1
+        if i % 64 == 0:
+            sync()
+    sync()
+    clocks = sampler.stop()
+    sparq.sparq_check()
+    if world > 1:
+        t = torch.tensor([ms_total], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * OPS_PER_STEP / (ms_step * 1e-3) / 1e12
+
+    # end to end: pinned host input -> device -> fused kernel -> uint8 result back on the host
+    x_host = torch.from_numpy(synth.activations(SEED, (NB, H, W, C), ZERO_FRAC, stream=10)).pin_memory()
+    y_host = torch.empty((NB, H, W, COUT), dtype=torch.uint8).pin_memory()
+
+    def e2e_step():
+        sparq.sparq_conv2d_nhwc_s8_host(x_host, wt, (STRIDE, STRIDE), (PAD, PAD), params, scale=scale, bias=bias,
+                                        relu=True, inv_out_scale=inv, u8_out=y_host)
+    e2e_steps = max(10, min(args.steps, 100))
+    for _ in range(3):
+        e2e_step()
+    sync(); barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    f1.record()
+    sync(); barrier()
+    e2e_ms = f0.elapsed_time(f1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * OPS_PER_STEP / (e2e_ms / e2e_steps * 1e-3) / 1e12
+
+    int8_peak = pk["bf16"] * INT8_OVER_BF16
+    per_launch_tops = OPS_PER_STEP / (ms_step * 1e-3) / 1e12
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {
+            "workload": "resnet18_conv3x3_b32_56x56x64_to_64_s1_p1 (vSPARQ n=4 5opt +R, scale+bias+ReLU+requant u8)",
+            "global_batch": NB * world, "zero_frac": ZERO_FRAC,
+            "l2": f"rotating {sets} input/output sets ({sets * (IN_BYTES + OUT_BYTES) >> 20} MiB) larger than the 126 MiB L2",
+            "parallelism": f"replicas x{world}, batch sharded, no collective",
+        },
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"]},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": IN_BYTES, "d2h_bytes_per_step": OUT_BYTES,
+                "steps": e2e_steps},
+        "gpu_launches": args.steps,
+        "roofline": {
+            "bound": "tensor", "achieved": per_launch_tops, "peak": int8_peak, "unit": "TOP/s",
+            "frac": per_launch_tops / int8_peak,
+            "traffic": None,
+            "kernel": "sparq_gemm_kernel<64,64,VSPARQ,4,round> (implicit-GEMM conv)",
+            "peak_source": f"{pk['source']} bf16 burst {pk['bf16']} TFLOP/s x {INT8_OVER_BF16} (nominal int8:bf16 ratio)",
+            "algorithmic_ops_per_launch": OPS_PER_STEP,
+            "algorithmic_bytes_per_launch": IN_BYTES + OUT_BYTES + WGT_BYTES,
+            "hbm_floor_ms": (IN_BYTES + OUT_BYTES + WGT_BYTES) / (pk["hbm"] * 1e9) * 1e3,
+        },
+    }
+    if rank == 0 and world == 1:
+        tops, dt, cores = cpu_baseline(4)
+        line["cpu_baseline"] = {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"4 of {NB} images of the same layer, {dt:.2f} s"}
+        if not args.no_extras:
+            del xs, outs
+            torch.cuda.empty_cache()
+            line["extra"] = extras(device, pk, 10)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

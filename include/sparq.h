@@ -124,12 +124,39 @@ SPARQ_API int sparq_gemm_s8(const uint8_t *A, int64_t lda, const int8_t *B, int6
  * Output pixel (img, ho, wo) is row (img*Ho + ho)*Wo + wo of the M x cout outputs, with
  * Ho = (h + 2*pad_h - r)/stride_h + 1 and Wo likewise.
  * Requirements (else SPARQ_ERR_UNSUPPORTED): x and wgt 16-byte aligned, c a multiple of
- * 16 (64 or a multiple of 128 when r*s > 1), r, s in 1..7, strides in 1..8,
- * pads < filter size. */
+ * 16 (of 64 unless the filter is 1x1 with unit stride and no padding), r, s in 1..7,
+ * strides in 1..8, pads < filter size, r*s*c <= 65536. */
 SPARQ_API int sparq_conv2d_nhwc_s8(const uint8_t *x, int n, int h, int w, int c,
                          const int8_t *wgt, int cout, int r, int s,
                          int stride_h, int stride_w, int pad_h, int pad_w,
                          const sparq_params *p, const sparq_epilogue *e, void *stream);
+
+/* ---- Host-buffer forms -----------------------------------------------------------------
+ * The same operations for callers whose activations live in HOST memory (pinned memory
+ * gives asynchronous copies; pageable memory works but is slower).  The library copies
+ * the input into a device staging buffer that it owns (grown on demand, kept for later
+ * calls, freed by sparq_shutdown), runs the device entry point on `stream`, copies the
+ * requested outputs back and SYNCHRONIZES `stream` before returning.  Calls that share a
+ * device share the staging buffers, so do not issue two host-buffer calls concurrently on
+ * one device.  Parameters (weights, scale, bias) stay DEVICE pointers: they are resident
+ * model data, not per-step inputs. */
+
+/* in_host / out_host: HOST pointers, rows * row_len bytes each (may be the same). */
+SPARQ_API int sparq_quantize_host(const uint8_t *in_host, uint8_t *out_host, size_t rows, size_t row_len,
+                        const sparq_params *p, void *stream);
+
+/* A_host: HOST, M x K with leading dimension lda.  B: DEVICE.  In `e`, scale and bias are
+ * DEVICE pointers and acc_out / f32_out / u8_out are HOST pointers (M x N each). */
+SPARQ_API int sparq_gemm_s8_host(const uint8_t *A_host, int64_t lda, const int8_t *B, int64_t ldb,
+                       int64_t M, int64_t N, int64_t K,
+                       const sparq_params *p, const sparq_epilogue *e, void *stream);
+
+/* x_host: HOST NHWC tensor.  wgt: DEVICE.  In `e`, scale and bias are DEVICE pointers and
+ * the output pointers are HOST pointers (n*Ho*Wo x cout each). */
+SPARQ_API int sparq_conv2d_nhwc_s8_host(const uint8_t *x_host, int n, int h, int w, int c,
+                              const int8_t *wgt, int cout, int r, int s,
+                              int stride_h, int stride_w, int pad_h, int pad_w,
+                              const sparq_params *p, const sparq_epilogue *e, void *stream);
 
 /* Synchronizes `stream` and reports what the device-side code recorded since the last
  * check: SPARQ_OK, SPARQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up (its

@@ -13,5 +13,6 @@ from ._binding import (  # noqa: F401
     SET_5OPT, SET_3OPT, SET_2OPT, SET_6OPT, SET_7OPT,
     library_path, load_library,
     sparq_quantize, sparq_gemm_s8, sparq_conv2d_nhwc_s8,
+    sparq_quantize_host, sparq_gemm_s8_host, sparq_conv2d_nhwc_s8_host,
     sparq_check, sparq_last_error, sparq_shutdown,
 )

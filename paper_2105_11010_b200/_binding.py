@@ -77,6 +77,12 @@ def load_library() -> ctypes.CDLL:
                                            i32, i32, i32, i32,
                                            ctypes.POINTER(_CParams), ctypes.POINTER(_CEpilogue), vp]
         L.sparq_conv2d_nhwc_s8.restype = i32
+        L.sparq_quantize_host.argtypes = L.sparq_quantize.argtypes
+        L.sparq_quantize_host.restype = i32
+        L.sparq_gemm_s8_host.argtypes = L.sparq_gemm_s8.argtypes
+        L.sparq_gemm_s8_host.restype = i32
+        L.sparq_conv2d_nhwc_s8_host.argtypes = L.sparq_conv2d_nhwc_s8.argtypes
+        L.sparq_conv2d_nhwc_s8_host.restype = i32
         L.sparq_check.argtypes = [vp]
         L.sparq_check.restype = i32
         L.sparq_last_error.argtypes = []
@@ -185,3 +191,74 @@ def sparq_conv2d_nhwc_s8(x: torch.Tensor, w: torch.Tensor, stride, pad, params: 
                                                _dev(w, torch.int8, "w"), cout, r, s,
                                                stride[0], stride[1], pad[0], pad[1],
                                                ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))
+
+
+# ---- host-buffer forms ------------------------------------------------------------------
+
+def _host(t: Optional[torch.Tensor], dtype, name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if t.is_cuda:
+        raise ValueError(f"{name} must be a CPU tensor (pinned for asynchronous copies)")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous {dtype} tensor")
+    return t.data_ptr() or None
+
+
+def sparq_quantize_host(inp: torch.Tensor, out: torch.Tensor, rows: int, row_len: int,
+                        params: SparqParams, stream=None) -> None:
+    """Host-buffer form of :func:`sparq_quantize`; returns after the result is in ``out``."""
+    if inp.numel() < rows * row_len or out.numel() < rows * row_len:
+        raise ValueError("tensor smaller than rows * row_len")
+    p = params._c()
+    _raise(load_library().sparq_quantize_host(_host(inp, torch.uint8, "inp"), _host(out, torch.uint8, "out"),
+                                              rows, row_len, ctypes.byref(p), _stream_ptr(stream)))
+
+
+def sparq_gemm_s8_host(A: torch.Tensor, B: torch.Tensor, params: SparqParams, *,
+                       scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                       relu: bool = False, inv_out_scale: float = 1.0,
+                       acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
+                       u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Host-buffer form of :func:`sparq_gemm_s8`: ``A`` and the outputs are CPU tensors."""
+    M, K = A.shape
+    N, K2 = B.shape
+    if K != K2:
+        raise ValueError("A and B disagree on K")
+    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out)):
+        if t is not None and t.numel() < M * N:
+            raise ValueError(f"{name} has fewer than M*N elements")
+    p = params._c()
+    e = _CEpilogue(_dev(scale, torch.float32, "scale"), _dev(bias, torch.float32, "bias"),
+                   int(bool(relu)), float(inv_out_scale),
+                   _host(acc_out, torch.int32, "acc_out"), _host(f32_out, torch.float32, "f32_out"),
+                   _host(u8_out, torch.uint8, "u8_out"))
+    _raise(load_library().sparq_gemm_s8_host(_host(A, torch.uint8, "A"), K, _dev(B, torch.int8, "B"), K,
+                                             M, N, K, ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))
+
+
+def sparq_conv2d_nhwc_s8_host(x: torch.Tensor, w: torch.Tensor, stride, pad, params: SparqParams, *,
+                              scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                              relu: bool = False, inv_out_scale: float = 1.0,
+                              acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
+                              u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Host-buffer form of :func:`sparq_conv2d_nhwc_s8`: ``x`` and the outputs are CPU tensors."""
+    nb, h, wd, c = x.shape
+    cout, r, s, c2 = w.shape
+    if c != c2:
+        raise ValueError("x and w disagree on the channel count")
+    ho = (h + 2 * pad[0] - r) // stride[0] + 1
+    wo = (wd + 2 * pad[1] - s) // stride[1] + 1
+    m = nb * ho * wo
+    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out)):
+        if t is not None and t.numel() < m * cout:
+            raise ValueError(f"{name} has fewer than N*Ho*Wo*Cout elements")
+    p = params._c()
+    e = _CEpilogue(_dev(scale, torch.float32, "scale"), _dev(bias, torch.float32, "bias"),
+                   int(bool(relu)), float(inv_out_scale),
+                   _host(acc_out, torch.int32, "acc_out"), _host(f32_out, torch.float32, "f32_out"),
+                   _host(u8_out, torch.uint8, "u8_out"))
+    _raise(load_library().sparq_conv2d_nhwc_s8_host(_host(x, torch.uint8, "x"), nb, h, wd, c,
+                                                    _dev(w, torch.int8, "w"), cout, r, s,
+                                                    stride[0], stride[1], pad[0], pad[1],
+                                                    ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))

@@ -95,7 +95,8 @@ int get_status_word(unsigned int **dptr)
     return SPARQ_OK;
 }
 
-void release_gemm_state();  // sparq_gemm.cu
+void release_gemm_state();     // sparq_gemm.cu
+void release_host_staging();   // sparq_host.cu
 
 }  // namespace sparq
 
@@ -129,6 +130,7 @@ extern "C" int sparq_check(void *stream)
 extern "C" int sparq_shutdown(void)
 {
     release_gemm_state();
+    release_host_staging();
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) {
         cudaGetLastError();
