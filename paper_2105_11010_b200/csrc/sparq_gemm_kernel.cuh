@@ -178,7 +178,23 @@ __device__ __forceinline__ constexpr uint32_t make_idesc_i8(int n)
     return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 }
 
-__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Barrier among the epilogue warps only (hardware barrier 1).
+__device__ __forceinline__ void epi_bar_sync()
+{
+    asm volatile("bar.sync 1, %0;" :: "n"(kNumEpiWarps * 32) : "memory");
+}
+
+// 32 contiguous bytes with one 256-bit store (dst 32-byte aligned).
+__device__ __forceinline__ void st_global_v8(void *dst, const uint32_t (&w)[8])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_32x32_issue(uint32_t taddr, uint32_t (&r)[32])
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -189,7 +205,6 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
 // ---- epilogue arithmetic ----------------------------------------------------------------
@@ -203,12 +218,21 @@ __device__ __forceinline__ float dequant(int32_t acc, float scale, float bias, i
     return y;
 }
 
-__device__ __forceinline__ uint32_t requant(float y, float inv_out_scale)
+// clamp(rint(y * inv_out_scale), 0, 255) without a float->int conversion: clamping to
+// [0, 255] first commutes with the rounding (both bounds are integers; NaN clamps to 0),
+// and adding 1.5 * 2^23 rounds to the nearest integer, ties to even, leaving that integer
+// in the low 8 bits of the float's bit pattern.
+__device__ __forceinline__ uint32_t requant_bits(float y, float inv_out_scale)
 {
-    float u = rintf(__fmul_rn(y, inv_out_scale));
-    if (!(u > 0.0f)) return 0u;          // negative, zero and NaN
-    if (u > 255.0f) return 255u;
-    return (uint32_t)u;
+    float z = __fmul_rn(y, inv_out_scale);
+    z = fminf(fmaxf(z, 0.0f), 255.0f);
+    return __float_as_uint(__fadd_rn(z, 12582912.0f));
+}
+
+// low bytes of four words -> one word
+__device__ __forceinline__ uint32_t pack4(uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    return prmt(prmt(a, b, 0x0040u), prmt(c, d, 0x0040u), 0x5410u);
 }
 
 // ---- the kernel ---------------------------------------------------------------------------
@@ -236,6 +260,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     __shared__ __align__(8) uint64_t bar_acc_full[2], bar_acc_empty[2], bar_done;
     __shared__ uint32_t tmem_base_slot;
     __shared__ uint32_t abort_word;
+    __shared__ __align__(16) float s_scale[BN], s_bias[BN];
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -352,21 +377,46 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     } else if (warp < kFirstXfWarp) {
         // ================= epilogue =================
         const int quarter = warp & 3;                   // tensor-memory lanes this warp may read
+        const int et = threadIdx.x - kFirstEpiWarp * 32;   // 0 .. 127
         uint32_t local_tile = 0;
-        const bool vec_ok = (g.N % 16) == 0;
+        const bool vec_ok = (g.N % 32) == 0;
+        const bool need_f = (g.f32_out != nullptr) || (g.u8_out != nullptr);
+        const bool u8_wide = (reinterpret_cast<uintptr_t>(g.u8_out) & 31u) == 0;   // 256-bit stores allowed
+        constexpr int kChunks = BN / 32;
         for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
             const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
             const int acc = local_tile & 1;
             const uint32_t acc_use = local_tile >> 1;
+            // per-column scale and bias of this tile, staged once in shared memory
+            if (need_f) {
+                epi_bar_sync();                             // previous tile's readers are done
+                for (int c = et; c < BN; c += kNumEpiWarps * 32) {
+                    const int64_t col = nt * BN + c;
+                    const bool ok = col < g.N;
+                    s_scale[c] = ok ? __ldg(g.scale + col) : 0.0f;
+                    s_bias[c] = (ok && g.bias) ? __ldg(g.bias + col) : 0.0f;
+                }
+                epi_bar_sync();
+            }
             mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status);
             tc_fence_after();
             const int64_t row = mt * kBM + quarter * 32 + lane;
             const bool row_ok = row < g.M;
-#pragma unroll 1
-            for (int ch = 0; ch < BN / 32; ++ch) {
-                uint32_t r[32];
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + ch * 32);
-                tmem_ld_32x32(taddr, r);
+            const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+            uint32_t r[2][32];
+            tmem_ld_32x32_issue(taddr0, r[0]);
+#pragma unroll
+            for (int ch = 0; ch < kChunks; ++ch) {
+                tmem_ld_wait();
+                if (ch + 1 < kChunks) {
+                    tmem_ld_32x32_issue(taddr0 + (uint32_t)((ch + 1) * 32), r[(ch + 1) & 1]);
+                } else {
+                    // the whole accumulator is in registers: hand it back to the MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
+                }
+                const uint32_t(&v)[32] = r[ch & 1];
                 const int64_t col0 = nt * BN + ch * 32;
                 if (!row_ok || col0 >= g.N) continue;
                 const int64_t off = row * g.N + col0;
@@ -375,27 +425,28 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     if (full) {
                         int4 *dst = reinterpret_cast<int4 *>(g.acc_out + off);
 #pragma unroll
-                        for (int v = 0; v < 8; ++v)
-                            dst[v] = make_int4((int)r[4 * v], (int)r[4 * v + 1], (int)r[4 * v + 2], (int)r[4 * v + 3]);
+                        for (int q = 0; q < 8; ++q)
+                            dst[q] = make_int4((int)v[4 * q], (int)v[4 * q + 1], (int)v[4 * q + 2], (int)v[4 * q + 3]);
                     } else {
-                        for (int i = 0; i < 32 && col0 + i < g.N; ++i) g.acc_out[off + i] = (int32_t)r[i];
+                        for (int i = 0; i < 32 && col0 + i < g.N; ++i) g.acc_out[off + i] = (int32_t)v[i];
                     }
                 }
-                if (g.f32_out || g.u8_out) {
+                if (need_f) {
                     float y[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int64_t c = col0 + i;
-                        const bool ok = c < g.N;
-                        const float sc = ok ? __ldg(g.scale + c) : 0.0f;
-                        const float bi = (ok && g.bias) ? __ldg(g.bias + c) : 0.0f;
-                        y[i] = dequant((int32_t)r[i], sc, bi, g.relu);
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 sc = *reinterpret_cast<const float4 *>(&s_scale[ch * 32 + 4 * q]);
+                        const float4 bi = *reinterpret_cast<const float4 *>(&s_bias[ch * 32 + 4 * q]);
+                        y[4 * q + 0] = dequant((int32_t)v[4 * q + 0], sc.x, bi.x, g.relu);
+                        y[4 * q + 1] = dequant((int32_t)v[4 * q + 1], sc.y, bi.y, g.relu);
+                        y[4 * q + 2] = dequant((int32_t)v[4 * q + 2], sc.z, bi.z, g.relu);
+                        y[4 * q + 3] = dequant((int32_t)v[4 * q + 3], sc.w, bi.w, g.relu);
                     }
                     if (g.f32_out) {
                         if (full) {
                             float4 *dst = reinterpret_cast<float4 *>(g.f32_out + off);
 #pragma unroll
-                            for (int v = 0; v < 8; ++v) dst[v] = make_float4(y[4 * v], y[4 * v + 1], y[4 * v + 2], y[4 * v + 3]);
+                            for (int q = 0; q < 8; ++q) dst[q] = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
                         } else {
                             for (int i = 0; i < 32 && col0 + i < g.N; ++i) g.f32_out[off + i] = y[i];
                         }
@@ -403,10 +454,12 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     if (g.u8_out) {
                         uint32_t w[8];
 #pragma unroll
-                        for (int v = 0; v < 8; ++v)
-                            w[v] = requant(y[4 * v], g.inv_out_scale) | (requant(y[4 * v + 1], g.inv_out_scale) << 8) |
-                                   (requant(y[4 * v + 2], g.inv_out_scale) << 16) | (requant(y[4 * v + 3], g.inv_out_scale) << 24);
-                        if (full) {
+                        for (int q = 0; q < 8; ++q)
+                            w[q] = pack4(requant_bits(y[4 * q], g.inv_out_scale), requant_bits(y[4 * q + 1], g.inv_out_scale),
+                                         requant_bits(y[4 * q + 2], g.inv_out_scale), requant_bits(y[4 * q + 3], g.inv_out_scale));
+                        if (full && u8_wide) {
+                            st_global_v8(g.u8_out + off, w);
+                        } else if (full) {
                             uint4 *dst = reinterpret_cast<uint4 *>(g.u8_out + off);
                             dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
                             dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
@@ -417,9 +470,6 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
         }
     } else if (MODE != SPARQ_MODE_NONE) {
         // ================= transform =================
