@@ -158,6 +158,38 @@ SPARQ_API int sparq_conv2d_nhwc_s8_host(const uint8_t *x_host, int n, int h, int
                               int stride_h, int stride_w, int pad_h, int pad_w,
                               const sparq_params *p, const sparq_epilogue *e, void *stream);
 
+/* ---- For callers that cannot allocate device memory ---------------------------------------
+ * (The paper has no counterpart: this is a deployment variant of sparq_gemm_s8.)
+ *
+ * Some hosts of this library must not call cudaMalloc once they are running: a serving
+ * process whose framework has already claimed all free device memory for its own pool
+ * (a later cudaMalloc fails or fragments the pool), or a control loop that cannot take
+ * the device-wide synchronization an allocation implies.  The other entry points
+ * allocate lazily (the status word, staging buffers); this one allocates nothing, on the
+ * host's behalf or through any library: no cudaMalloc, no cudaFree, no torch allocator.
+ *
+ * It computes exactly what sparq_gemm_s8 computes, as two kernels: the standalone
+ * transform writes T(A) into scratch, then the plain u8 x s8 GEMM with the same epilogue
+ * reads it.  The scratch (and the status word of the bounded waits) lives in a fixed
+ * array inside the library image, SPARQ_STATIC_SCRATCH_BYTES long, which every GPU that
+ * loads the library holds until the process exits.
+ *
+ *   - Limit: M * K <= SPARQ_STATIC_SCRATCH_BYTES and lda == K; anything larger returns
+ *     SPARQ_ERR_UNSUPPORTED with the limit in sparq_last_error().  Other requirements as
+ *     for sparq_gemm_s8.
+ *   - The first call on a device looks up the array's device address (set-up, once per
+ *     device, with that device current).  Make that first call outside any stream capture.
+ *   - The call is synchronous: it returns after `stream` has drained, so the outputs are
+ *     complete and a device-side timeout is reported by this call (SPARQ_ERR_TIMEOUT),
+ *     not by sparq_check.
+ *   - All calls share the one array, which keeps the previous call's contents.  Calls that
+ *     overlap on the GPU (other host threads, other streams, other processes' contexts do
+ *     not count) race on it: issue them one at a time per device. */
+#define SPARQ_STATIC_SCRATCH_BYTES (8u << 20)
+SPARQ_API int sparq_gemm_s8_static(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                         int64_t M, int64_t N, int64_t K,
+                         const sparq_params *p, const sparq_epilogue *e, void *stream);
+
 /* Synchronizes `stream` and reports what the device-side code recorded since the last
  * check: SPARQ_OK, SPARQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up (its
  * outputs are then undefined), or SPARQ_ERR_CUDA if the stream is in error. */

@@ -83,6 +83,8 @@ def load_library() -> ctypes.CDLL:
         L.sparq_gemm_s8_host.restype = i32
         L.sparq_conv2d_nhwc_s8_host.argtypes = L.sparq_conv2d_nhwc_s8.argtypes
         L.sparq_conv2d_nhwc_s8_host.restype = i32
+        L.sparq_gemm_s8_static.argtypes = L.sparq_gemm_s8.argtypes
+        L.sparq_gemm_s8_static.restype = i32
         L.sparq_check.argtypes = [vp]
         L.sparq_check.restype = i32
         L.sparq_last_error.argtypes = []
@@ -262,3 +264,31 @@ def sparq_conv2d_nhwc_s8_host(x: torch.Tensor, w: torch.Tensor, stride, pad, par
                                                     _dev(w, torch.int8, "w"), cout, r, s,
                                                     stride[0], stride[1], pad[0], pad[1],
                                                     ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def sparq_gemm_s8_static(A: torch.Tensor, B: torch.Tensor, params: SparqParams, *,
+                         scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                         relu: bool = False, inv_out_scale: float = 1.0,
+                         acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
+                         u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """``sparq_gemm_s8`` for hosts that must not allocate device memory once running
+    (all free memory already belongs to a framework's pool, or an allocation's
+    device-wide synchronization is not acceptable).  Same result, computed as transform
+    kernel + plain GEMM with the transformed activations in a fixed scratch array inside
+    the library (``M * K <= STATIC_SCRATCH_BYTES``).  Synchronous; one call at a time per
+    device.  The first call on a device performs the address look-up: make it before any
+    stream capture."""
+    M, K = A.shape
+    N, K2 = B.shape
+    if K != K2:
+        raise ValueError("A and B disagree on K")
+    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out)):
+        if t is not None and t.numel() < M * N:
+            raise ValueError(f"{name} has fewer than M*N elements")
+    p = params._c()
+    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out)
+    _raise(load_library().sparq_gemm_s8_static(_dev(A, torch.uint8, "A"), K, _dev(B, torch.int8, "B"), K,
+                                               M, N, K, ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))

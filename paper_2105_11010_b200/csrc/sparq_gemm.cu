@@ -169,6 +169,36 @@ static int gemm_impl(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     return SPARQ_OK;
 }
 
+// The same launch as gemm_impl for callers that bring their own status word (a device
+// pointer) instead of the library-allocated one.  Nothing here allocates device memory.
+int gemm_with_status(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb, int64_t M, int64_t N, int64_t K,
+                     const XformArgs &x, const sparq_epilogue *e, unsigned int *status, cudaStream_t st)
+{
+    int sms = 0;
+    int rc = device_info(&sms);
+    if (rc != SPARQ_OK) return rc;
+    const int64_t pad128 = (K + 127) / 128 * 128, pad64 = (K + 63) / 64 * 64;
+    const int bk = (pad64 < pad128) ? 64 : 128;
+    const int bn = pick_bn(M, N, sms);
+    CUtensorMap ma, mb;
+    rc = encode_2d(&ma, A, K, M, lda, bk, kBM);
+    if (rc != SPARQ_OK) return rc;
+    rc = encode_2d(&mb, B, K, N, ldb, bk, bn);
+    if (rc != SPARQ_OK) return rc;
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.M = M; g.N = N; g.K = K;
+    g.k_blocks = (int)((K + bk - 1) / bk);
+    fill_common(&g, x, e, status);
+    const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
+    if (ce != cudaSuccess) return cuda_error(ce, "sparq_gemm_kernel launch");
+    return SPARQ_OK;
+}
+
+int check_epilogue_args(const sparq_epilogue *e) { return check_epilogue(e); }
+
 }  // namespace sparq
 
 using namespace sparq;
