@@ -7,9 +7,10 @@
 //                 convolution) and B tile into a ring of shared-memory stages
 //   warp 1        allocates tensor memory; one lane issues tcgen05.mma kind::i8
 //                 (u8 x s8 -> s32) on each transformed stage
-//   warps 2..5    epilogue: tcgen05.ld of a finished accumulator, fp32 scale / bias /
-//                 ReLU / requantize, global stores
-//   warps 6..13   transform: rewrite the A stage in place with bSPARQ / vSPARQ
+//   warps 2..9    epilogue: tcgen05.ld of a finished accumulator, fp32 scale / bias /
+//                 ReLU / requantize, global stores (warp w reads lane quarter w % 4 and
+//                 one half of the tile's columns)
+//   warps 10..17  transform: rewrite the A stage in place with bSPARQ / vSPARQ
 //
 // A stage travels  TMA (async proxy) -> transform warps (generic proxy) -> MMA (async
 // proxy); the hand-offs are mbarriers, with fence.proxy.async after the in-place rewrite.
@@ -30,7 +31,7 @@
 namespace sparq {
 
 constexpr int kBM = 128;                 // rows of an output tile = MMA M
-constexpr int kNumEpiWarps = 4;
+constexpr int kNumEpiWarps = 8;          // two per tensor-memory lane quarter
 constexpr int kNumXfWarps = 8;
 constexpr int kFirstEpiWarp = 2;
 constexpr int kFirstXfWarp = kFirstEpiWarp + kNumEpiWarps;
@@ -209,12 +210,15 @@ __device__ __forceinline__ void tmem_ld_32x32_issue(uint32_t taddr, uint32_t (&r
 
 // ---- epilogue arithmetic ----------------------------------------------------------------
 
-// int32 accumulator -> (fp32 value, requantized byte), one IEEE operation per step.
+// int32 accumulator -> fp32 value, one IEEE operation per step.  SMALL: the caller
+// guarantees |acc| < 2^22, where (float)acc is exact and equals
+// bits(acc + bits(1.5 * 2^23)) - 1.5 * 2^23.
+template <bool SMALL>
 __device__ __forceinline__ float dequant(int32_t acc, float scale, float bias, int relu)
 {
-    float t = __int2float_rn(acc);
+    float t = SMALL ? __fadd_rn(__int_as_float(acc + 0x4B400000), -12582912.0f) : __int2float_rn(acc);
     float y = __fmaf_rn(t, scale, bias);
-    if (relu) y = (y > 0.0f) ? y : 0.0f;
+    if (relu) y = fmaxf(y, 0.0f);        // NaN -> 0, like (y > 0 ? y : 0)
     return y;
 }
 
@@ -376,19 +380,28 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         __syncwarp();
     } else if (warp < kFirstXfWarp) {
         // ================= epilogue =================
-        const int quarter = warp & 3;                   // tensor-memory lanes this warp may read
-        const int et = threadIdx.x - kFirstEpiWarp * 32;   // 0 .. 127
+        const int quarter = warp & 3;                        // tensor-memory lanes this warp may read
+        const int half = (warp - kFirstEpiWarp) >> 2;        // which half of the tile's columns
+        const int et = threadIdx.x - kFirstEpiWarp * 32;     // 0 .. 255
         uint32_t local_tile = 0;
         const bool vec_ok = (g.N % 32) == 0;
         const bool need_f = (g.f32_out != nullptr) || (g.u8_out != nullptr);
         const bool u8_wide = (reinterpret_cast<uintptr_t>(g.u8_out) & 31u) == 0;   // 256-bit stores allowed
-        constexpr int kChunks = BN / 32;
+        // relu(y) * inv clamped to [0, 255] equals y * inv clamped when inv > 0, so the
+        // ReLU select is only needed when the fp32 value itself is an output
+        const bool relu_op = g.relu && (g.f32_out != nullptr || !(g.inv_out_scale > 0.0f));
+        // |acc| <= K * 255 * 128; below 2^22 the int -> float conversion is exact and can be
+        // done with an integer add and a float subtract instead of the conversion unit
+        const bool small_acc = g.K * (255 * 128) < (1 << 22);
+        constexpr int kChunks = BN / 64;                     // 32-column chunks per warp
+        int64_t staged_nt = -1;
         for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
             const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
             const int acc = local_tile & 1;
             const uint32_t acc_use = local_tile >> 1;
-            // per-column scale and bias of this tile, staged once in shared memory
-            if (need_f) {
+            // per-column scale and bias, staged in shared memory whenever the column tile changes
+            if (need_f && nt != staged_nt) {
+                staged_nt = nt;
                 epi_bar_sync();                             // previous tile's readers are done
                 for (int c = et; c < BN; c += kNumEpiWarps * 32) {
                     const int64_t col = nt * BN + c;
@@ -402,22 +415,21 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             tc_fence_after();
             const int64_t row = mt * kBM + quarter * 32 + lane;
             const bool row_ok = row < g.M;
-            const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
-            uint32_t r[2][32];
-            tmem_ld_32x32_issue(taddr0, r[0]);
-#pragma unroll
+            const int cbase = half * (BN / 2);
+            const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + cbase);
+#pragma unroll 1
             for (int ch = 0; ch < kChunks; ++ch) {
+                uint32_t v[32];
+                tmem_ld_32x32_issue(taddr0 + (uint32_t)(ch * 32), v);
                 tmem_ld_wait();
-                if (ch + 1 < kChunks) {
-                    tmem_ld_32x32_issue(taddr0 + (uint32_t)((ch + 1) * 32), r[(ch + 1) & 1]);
-                } else {
-                    // the whole accumulator is in registers: hand it back to the MMA warp
+                if (ch + 1 == kChunks) {
+                    // this warp's share of the accumulator is in registers: hand it back
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
                 }
-                const uint32_t(&v)[32] = r[ch & 1];
-                const int64_t col0 = nt * BN + ch * 32;
+                const int ct = cbase + ch * 32;              // column inside the tile
+                const int64_t col0 = nt * BN + ct;
                 if (!row_ok || col0 >= g.N) continue;
                 const int64_t off = row * g.N + col0;
                 const bool full = vec_ok && (col0 + 32 <= g.N);
@@ -432,31 +444,40 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     }
                 }
                 if (need_f) {
-                    float y[32];
+                    // v[i] becomes the fp32 value's bits in place
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
-                        const float4 sc = *reinterpret_cast<const float4 *>(&s_scale[ch * 32 + 4 * q]);
-                        const float4 bi = *reinterpret_cast<const float4 *>(&s_bias[ch * 32 + 4 * q]);
-                        y[4 * q + 0] = dequant((int32_t)v[4 * q + 0], sc.x, bi.x, g.relu);
-                        y[4 * q + 1] = dequant((int32_t)v[4 * q + 1], sc.y, bi.y, g.relu);
-                        y[4 * q + 2] = dequant((int32_t)v[4 * q + 2], sc.z, bi.z, g.relu);
-                        y[4 * q + 3] = dequant((int32_t)v[4 * q + 3], sc.w, bi.w, g.relu);
+                        const float4 sc = *reinterpret_cast<const float4 *>(&s_scale[ct + 4 * q]);
+                        const float4 bi = *reinterpret_cast<const float4 *>(&s_bias[ct + 4 * q]);
+                        if (small_acc) {
+                            v[4 * q + 0] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 0], sc.x, bi.x, relu_op));
+                            v[4 * q + 1] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 1], sc.y, bi.y, relu_op));
+                            v[4 * q + 2] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 2], sc.z, bi.z, relu_op));
+                            v[4 * q + 3] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 3], sc.w, bi.w, relu_op));
+                        } else {
+                            v[4 * q + 0] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 0], sc.x, bi.x, relu_op));
+                            v[4 * q + 1] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 1], sc.y, bi.y, relu_op));
+                            v[4 * q + 2] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 2], sc.z, bi.z, relu_op));
+                            v[4 * q + 3] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 3], sc.w, bi.w, relu_op));
+                        }
                     }
                     if (g.f32_out) {
                         if (full) {
-                            float4 *dst = reinterpret_cast<float4 *>(g.f32_out + off);
+                            uint4 *dst = reinterpret_cast<uint4 *>(g.f32_out + off);
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) dst[q] = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+                            for (int q = 0; q < 8; ++q) dst[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
                         } else {
-                            for (int i = 0; i < 32 && col0 + i < g.N; ++i) g.f32_out[off + i] = y[i];
+                            for (int i = 0; i < 32 && col0 + i < g.N; ++i) g.f32_out[off + i] = __uint_as_float(v[i]);
                         }
                     }
                     if (g.u8_out) {
                         uint32_t w[8];
 #pragma unroll
                         for (int q = 0; q < 8; ++q)
-                            w[q] = pack4(requant_bits(y[4 * q], g.inv_out_scale), requant_bits(y[4 * q + 1], g.inv_out_scale),
-                                         requant_bits(y[4 * q + 2], g.inv_out_scale), requant_bits(y[4 * q + 3], g.inv_out_scale));
+                            w[q] = pack4(requant_bits(__uint_as_float(v[4 * q]), g.inv_out_scale),
+                                         requant_bits(__uint_as_float(v[4 * q + 1]), g.inv_out_scale),
+                                         requant_bits(__uint_as_float(v[4 * q + 2]), g.inv_out_scale),
+                                         requant_bits(__uint_as_float(v[4 * q + 3]), g.inv_out_scale));
                         if (full && u8_wide) {
                             st_global_v8(g.u8_out + off, w);
                         } else if (full) {
@@ -473,7 +494,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
     } else if (MODE != SPARQ_MODE_NONE) {
         // ================= transform =================
-        const int xt = threadIdx.x - kFirstXfWarp * 32;            // 0 .. 255
+        const int xt = threadIdx.x - kFirstXfWarp * 32;            // 0 .. 255 among the transform threads
         constexpr int kXfThreads = kNumXfWarps * 32;
         constexpr int kVecs = Cfg::kABytes / 16;
         constexpr int kPerThread = kVecs / kXfThreads;
@@ -526,9 +547,16 @@ cudaError_t launch_gemm_shape(const CUtensorMap &ma, const CUtensorMap &mb, cons
 #define SPARQ_LAUNCH_VARIANT(MODE_, XN_, RND_)                                                         \
     do {                                                                                               \
         auto kfn = sparq_gemm_kernel<BN, BK, MODE_, XN_, RND_>;                                        \
-        cudaError_t e_ = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
-                                              TileCfg<BN, BK>::kSmemBytes);                            \
+        static bool attr_set[64] = {};   /* per device ordinal */                                     \
+        int dev_ = 0;                                                                                  \
+        cudaError_t e_ = cudaGetDevice(&dev_);                                                         \
         if (e_ != cudaSuccess) return e_;                                                              \
+        if (dev_ < 0 || dev_ >= 64 || !attr_set[dev_]) {                                               \
+            e_ = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize,                \
+                                      TileCfg<BN, BK>::kSmemBytes);                                    \
+            if (e_ != cudaSuccess) return e_;                                                          \
+            if (dev_ >= 0 && dev_ < 64) attr_set[dev_] = true;                                         \
+        }                                                                                              \
         kfn<<<grid, kGemmThreads, TileCfg<BN, BK>::kSmemBytes, st>>>(ma, mb, g);                       \
         return cudaGetLastError();                                                                     \
     } while (0)
