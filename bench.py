@@ -135,6 +135,33 @@ def time_region(fn, steps, warmup, sync):
     return e0.elapsed_time(e1)      # ms
 
 
+def transform_section(device, pk, n, steps, warmup):
+    """Standalone transform on n uint8 activations (50 % zeros), bSPARQ and vSPARQ, n = 4,
+    five placements, round to nearest; rows of 1024.  Bytes = n read + n written."""
+    import torch
+    import paper_2105_11010_b200 as sparq
+    sync = torch.cuda.synchronize
+    gen = torch.Generator(device=device).manual_seed(4)
+    x = torch.empty(n, dtype=torch.uint8, device=device)
+    chunk = min(n, 1 << 26)
+    for lo in range(0, n, chunk):
+        z = torch.randn(chunk, generator=gen, device=device)
+        v = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
+        v[torch.rand(chunk, generator=gen, device=device) < 0.5] = 0
+        x[lo:lo + chunk] = v
+    y = torch.empty_like(x)
+    tr = {"activations": n}
+    for name, mode in (("bsparq", sparq.MODE_BSPARQ), ("vsparq", sparq.MODE_VSPARQ)):
+        p = sparq.SparqParams(mode, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+        ms = time_region(lambda i: sparq.sparq_quantize(x, y, n // 1024, 1024, p), steps, warmup, sync) / steps
+        gbs = 2 * n / ms / 1e6
+        tr[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1),
+                    "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
+                                 "frac": round(gbs / pk["hbm"], 4), "traffic": None,
+                                 "peak_source": pk["source"] + " copy"}}
+    return tr
+
+
 def extras(device, pk, steps):
     """Other workloads of the same library, each with its own roofline: the standalone
     transform on 2^30 activations and the ResNet-50 layer sweep at batch 64."""
@@ -142,28 +169,7 @@ def extras(device, pk, steps):
     import paper_2105_11010_b200 as sparq
     out = {}
     sync = torch.cuda.synchronize
-    # --- standalone transform: 2^30 uint8 in, 2^30 out, 50 % zeros ---
-    n = 1 << 30
-    gen = torch.Generator(device=device).manual_seed(4)
-    x = torch.empty(n, dtype=torch.uint8, device=device)
-    chunk = 1 << 26
-    for lo in range(0, n, chunk):
-        z = torch.randn(chunk, generator=gen, device=device)
-        v = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
-        v[torch.rand(chunk, generator=gen, device=device) < 0.5] = 0
-        x[lo:lo + chunk] = v
-    y = torch.empty_like(x)
-    tr = {}
-    for name, mode in (("bsparq", sparq.MODE_BSPARQ), ("vsparq", sparq.MODE_VSPARQ)):
-        p = sparq.SparqParams(mode, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
-        ms = time_region(lambda i: sparq.sparq_quantize(x, y, 1 << 20, 1024, p), 20, 3, sync) / 20
-        gbs = 2 * n / ms / 1e6
-        tr[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1),
-                    "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
-                                 "frac": round(gbs / pk["hbm"], 4), "traffic": None,
-                                 "peak_source": pk["source"] + " copy"}}
-    out["transform_2p30"] = tr
-    del x, y
+    out["transform_2p30"] = transform_section(device, pk, 1 << 30, 20, 3)
     # --- ResNet-50 sweep, batch 64, every conv shape (22 shapes, 52 instances) ---
     p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
     layers, total_ms, total_ops = [], 0.0, 0
@@ -251,6 +257,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the transform and ResNet-50 sweep sections")
+    ap.add_argument("--section", default="main", choices=["main", "transform"],
+                    help="'transform' times only the standalone transform kernel (small, for profiling)")
+    ap.add_argument("--log2n", type=int, default=28, help="activations for --section transform (2^log2n)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
@@ -281,6 +290,9 @@ def main():
         torch.cuda.synchronize()
 
     pk = peaks()
+    if args.section == "transform":
+        print(json.dumps(transform_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
+        return
     sets = 20   # 20 x (6.4 MB in + 6.4 MB out) = 257 MB > 126 MB of L2
     xs, outs, wt, scale, bias = build_layer(device, sets)
     inv = synth.inv_out_scale(R * S * C, ZERO_FRAC)
