@@ -4,7 +4,7 @@
 
 #include <cstring>
 
-#include "sparq_gemm_kernel.cuh"
+#include "sparq_conv_window_kernel.cuh"
 
 namespace sparq {
 
@@ -169,6 +169,106 @@ static int gemm_impl(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     return SPARQ_OK;
 }
 
+// NHWC activation tensor read as a box of cb channels x wp columns x rows input rows of one
+// image (zero fill outside the image).
+static int encode_window(CUtensorMap *map, const void *ptr, int n, int h, int w, int c, int cb, int wp, int rows)
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        int rc = driver_fn("cuTensorMapEncodeTiled", (void **)&fn);
+        if (rc != SPARQ_OK) return rc;
+    }
+    cuuint64_t dims[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
+    cuuint64_t strides[3] = {(cuuint64_t)c, (cuuint64_t)c * w, (cuuint64_t)c * w * h};
+    cuuint32_t box[4] = {(cuuint32_t)cb, (cuuint32_t)wp, (cuuint32_t)rows, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(cb), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return set_error(SPARQ_ERR_CUDA, "cuTensorMapEncodeTiled (window) failed with CUresult %d", (int)r);
+    return SPARQ_OK;
+}
+
+constexpr int kMaxDynSmem = kWindowMaxDynSmem;
+
+// Stride-1 filters larger than 1x1: the window kernel, when its tiling fits.  Returns
+// 1 if it launched, 0 if the shape should take the im2col kernel, < 0 on error.
+static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, const int8_t *wgt, int cout, int r, int s,
+                           int pad_h, int pad_w, int ho, int wo, const XformArgs &x, const sparq_epilogue *e,
+                           int sms, unsigned int *status, cudaStream_t st)
+{
+    const int wp = w + 2 * pad_w;
+    if (wp > 128 || wo < 1) return 0;
+    const int cb = (c % 128 == 0) ? 128 : (c == 64 ? 64 : 0);
+    if (!cb) return 0;
+    int tr = 128 / wp;
+    if (tr > ho) tr = ho;
+    if (tr < 1 || tr * wo < 64) return 0;               // less than half of the MMA rows would be useful
+    const int c_blocks = c / cb;
+    const int taps = r * s;
+    const int kb_count = taps * c_blocks;
+    const int rows_alloc = (r - 1) * wp + (s - 1) + 128;
+    const int plane_bytes = (rows_alloc * cb + 1023) / 1024 * 1024;
+    const int win_bytes = plane_bytes * c_blocks;
+    const int tiles_per_img = (ho + tr - 1) / tr;
+    const int64_t m_tiles = (int64_t)n * tiles_per_img;
+
+    int bn;
+    if (cb == 64) {
+        if (cout > 64) return 0;
+        bn = 64;
+    } else {
+        if (cout <= 64) return 0;
+        bn = (cout > 128 && m_tiles * ((cout + 255) / 256) >= sms) ? 256 : 128;
+    }
+    const int b_block = bn * cb;
+    const int n_tiles = (cout + bn - 1) / bn;
+    bool resident = false;
+    int win_bufs = 2, b_stages = 0;
+    if (bn != 256 && n_tiles == 1 && 1024 + 2 * win_bytes + kb_count * b_block <= kMaxDynSmem) {
+        resident = true;
+        b_stages = kb_count;
+        if (1024 + 3 * win_bytes + kb_count * b_block <= kMaxDynSmem) win_bufs = 3;
+    } else {
+        if (bn == 64) return 0;                          // only the resident form is built for 64-wide tiles
+        const int left = kMaxDynSmem - 1024 - 2 * win_bytes;
+        b_stages = left / b_block;
+        if (b_stages > kMaxBStages) b_stages = kMaxBStages;
+        if (b_stages < 2) return 0;
+    }
+    const int smem_bytes = 1024 + win_bufs * win_bytes + b_stages * b_block;
+
+    CUtensorMap mx, mw;
+    int rc = encode_window(&mx, x_in, n, h, w, c, cb, wp, tr + r - 1);
+    if (rc != SPARQ_OK) return rc;
+    const int64_t K = (int64_t)r * s * c;
+    rc = encode_2d(&mw, wgt, K, cout, K, cb, bn);
+    if (rc != SPARQ_OK) return rc;
+
+    WindowArgs g;
+    memset(&g, 0, sizeof(g));
+    g.N = cout; g.K = K;
+    g.n_img = n; g.H = h; g.W = w; g.C = c; g.R = r; g.S = s; g.pad_h = pad_h; g.pad_w = pad_w; g.Ho = ho; g.Wo = wo;
+    g.Wp = wp; g.TR = tr; g.tiles_per_img = tiles_per_img; g.c_blocks = c_blocks;
+    g.box_bytes = cb * wp * (tr + r - 1);
+    g.plane_bytes = plane_bytes;
+    g.win_bufs = win_bufs;
+    g.b_stages = b_stages;
+    g.xf = XformDev{x.widen_c, x.widen_rounds, x.n};
+    g.scale = e->scale; g.bias = e->bias; g.relu = e->relu ? 1 : 0; g.inv_out_scale = e->inv_out_scale;
+    g.acc_out = e->acc_out; g.f32_out = e->f32_out; g.u8_out = e->u8_out;
+    g.status = status;
+    const int64_t tiles = m_tiles * n_tiles;
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    cudaError_t ce;
+    if (bn == 64) ce = launch_window_shape<64, 64, true>(mx, mw, g, x.mode, x.n, x.rnd, grid, smem_bytes, st);
+    else if (bn == 128 && resident) ce = launch_window_shape<128, 128, true>(mx, mw, g, x.mode, x.n, x.rnd, grid, smem_bytes, st);
+    else if (bn == 128) ce = launch_window_shape<128, 128, false>(mx, mw, g, x.mode, x.n, x.rnd, grid, smem_bytes, st);
+    else ce = launch_window_shape<256, 128, false>(mx, mw, g, x.mode, x.n, x.rnd, grid, smem_bytes, st);
+    if (ce != cudaSuccess) return cuda_error(ce, "sparq_conv_window_kernel launch");
+    return 1;
+}
+
 // The same launch as gemm_impl for callers that bring their own status word (a device
 // pointer) instead of the library-allocated one.  Nothing here allocates device memory.
 int gemm_with_status(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb, int64_t M, int64_t N, int64_t K,
@@ -261,6 +361,10 @@ extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, in
     unsigned int *status = nullptr;
     rc = get_status_word(&status);
     if (rc != SPARQ_OK) return rc;
+    if (stride_h == 1 && stride_w == 1) {
+        rc = try_window_conv(x_in, n, h, w, c, wgt, cout, r, s, pad_h, pad_w, ho, wo, x, e, sms, status, st);
+        if (rc != 0) return rc < 0 ? rc : SPARQ_OK;
+    }
     const int bk = (c % 128 == 0) ? 128 : 64;
     const int bn = pick_bn(M, cout, sms);
     CUtensorMap ma, mb;

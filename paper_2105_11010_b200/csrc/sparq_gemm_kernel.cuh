@@ -239,6 +239,122 @@ __device__ __forceinline__ uint32_t pack4(uint32_t a, uint32_t b, uint32_t c, ui
     return prmt(prmt(a, b, 0x0040u), prmt(c, d, 0x0040u), 0x5410u);
 }
 
+// Per-thread view of the epilogue's outputs and constants.
+struct EpiView {
+    int64_t N;
+    int32_t *acc_out;
+    float *f32_out;
+    uint8_t *u8_out;
+    float inv_out_scale;
+    bool need_f;      // a dequantized output is requested
+    bool relu_op;     // the ReLU select has to be executed (see below)
+    bool small_acc;   // |acc| < 2^22 guaranteed
+    bool vec_ok;      // rows allow 16/32-byte vector stores
+    bool u8_wide;     // 256-bit stores allowed on u8_out
+};
+
+template <class Args>
+__device__ __forceinline__ EpiView make_epi_view(const Args &g)
+{
+    EpiView e;
+    e.N = g.N;
+    e.acc_out = g.acc_out;
+    e.f32_out = g.f32_out;
+    e.u8_out = g.u8_out;
+    e.inv_out_scale = g.inv_out_scale;
+    e.need_f = (g.f32_out != nullptr) || (g.u8_out != nullptr);
+    // relu(y) * inv clamped to [0, 255] equals y * inv clamped when inv > 0, so the ReLU
+    // select is only needed when the fp32 value itself is an output
+    e.relu_op = g.relu && (g.f32_out != nullptr || !(g.inv_out_scale > 0.0f));
+    // |acc| <= K * 255 * 128; below 2^22 the int -> float conversion is exact and can be
+    // done with an integer add and a float subtract instead of the conversion unit
+    e.small_acc = g.K * (255 * 128) < (1 << 22);
+    e.vec_ok = (g.N % 32) == 0;
+    e.u8_wide = (reinterpret_cast<uintptr_t>(g.u8_out) & 31u) == 0;
+    return e;
+}
+
+// One thread's 32 consecutive accumulators of output row `row` (columns col0 .. col0+31,
+// tile-local column ct): optional raw store, dequantize, optional fp32 store, requantize
+// and store.  v is overwritten.
+__device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[32], int64_t row, int64_t col0, int ct,
+                                          const float *s_scale, const float *s_bias)
+{
+    const int64_t off = row * e.N + col0;
+    const bool full = e.vec_ok && (col0 + 32 <= e.N);
+    if (e.acc_out) {
+        if (full) {
+            int4 *dst = reinterpret_cast<int4 *>(e.acc_out + off);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                dst[q] = make_int4((int)v[4 * q], (int)v[4 * q + 1], (int)v[4 * q + 2], (int)v[4 * q + 3]);
+        } else {
+            for (int i = 0; i < 32 && col0 + i < e.N; ++i) e.acc_out[off + i] = (int32_t)v[i];
+        }
+    }
+    if (!e.need_f) return;
+    // v[i] becomes the fp32 value's bits in place
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const float4 sc = *reinterpret_cast<const float4 *>(&s_scale[ct + 4 * q]);
+        const float4 bi = *reinterpret_cast<const float4 *>(&s_bias[ct + 4 * q]);
+        if (e.small_acc) {
+            v[4 * q + 0] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 0], sc.x, bi.x, e.relu_op));
+            v[4 * q + 1] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 1], sc.y, bi.y, e.relu_op));
+            v[4 * q + 2] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 2], sc.z, bi.z, e.relu_op));
+            v[4 * q + 3] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 3], sc.w, bi.w, e.relu_op));
+        } else {
+            v[4 * q + 0] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 0], sc.x, bi.x, e.relu_op));
+            v[4 * q + 1] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 1], sc.y, bi.y, e.relu_op));
+            v[4 * q + 2] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 2], sc.z, bi.z, e.relu_op));
+            v[4 * q + 3] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 3], sc.w, bi.w, e.relu_op));
+        }
+    }
+    if (e.f32_out) {
+        if (full) {
+            uint4 *dst = reinterpret_cast<uint4 *>(e.f32_out + off);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) dst[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        } else {
+            for (int i = 0; i < 32 && col0 + i < e.N; ++i) e.f32_out[off + i] = __uint_as_float(v[i]);
+        }
+    }
+    if (e.u8_out) {
+        uint32_t w[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            w[q] = pack4(requant_bits(__uint_as_float(v[4 * q]), e.inv_out_scale),
+                         requant_bits(__uint_as_float(v[4 * q + 1]), e.inv_out_scale),
+                         requant_bits(__uint_as_float(v[4 * q + 2]), e.inv_out_scale),
+                         requant_bits(__uint_as_float(v[4 * q + 3]), e.inv_out_scale));
+        if (full && e.u8_wide) {
+            st_global_v8(e.u8_out + off, w);
+        } else if (full) {
+            uint4 *dst = reinterpret_cast<uint4 *>(e.u8_out + off);
+            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        } else {
+            for (int i = 0; i < 32 && col0 + i < e.N; ++i)
+                e.u8_out[off + i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
+        }
+    }
+}
+
+// Stages the scale and bias of columns n0 .. n0+bn-1 in shared memory (epilogue warps only).
+template <class Args>
+__device__ __forceinline__ void epi_stage_scale_bias(const Args &g, int64_t n0, int bn, int et,
+                                                     float *s_scale, float *s_bias)
+{
+    epi_bar_sync();                             // previous readers are done
+    for (int c = et; c < bn; c += kNumEpiWarps * 32) {
+        const int64_t col = n0 + c;
+        const bool ok = col < g.N;
+        s_scale[c] = ok ? __ldg(g.scale + col) : 0.0f;
+        s_bias[c] = (ok && g.bias) ? __ldg(g.bias + col) : 0.0f;
+    }
+    epi_bar_sync();
+}
+
 // ---- the kernel ---------------------------------------------------------------------------
 
 template <int BN, int BK>
@@ -383,33 +499,17 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const int quarter = warp & 3;                        // tensor-memory lanes this warp may read
         const int half = (warp - kFirstEpiWarp) >> 2;        // which half of the tile's columns
         const int et = threadIdx.x - kFirstEpiWarp * 32;     // 0 .. 255
+        const EpiView ev = make_epi_view(g);
         uint32_t local_tile = 0;
-        const bool vec_ok = (g.N % 32) == 0;
-        const bool need_f = (g.f32_out != nullptr) || (g.u8_out != nullptr);
-        const bool u8_wide = (reinterpret_cast<uintptr_t>(g.u8_out) & 31u) == 0;   // 256-bit stores allowed
-        // relu(y) * inv clamped to [0, 255] equals y * inv clamped when inv > 0, so the
-        // ReLU select is only needed when the fp32 value itself is an output
-        const bool relu_op = g.relu && (g.f32_out != nullptr || !(g.inv_out_scale > 0.0f));
-        // |acc| <= K * 255 * 128; below 2^22 the int -> float conversion is exact and can be
-        // done with an integer add and a float subtract instead of the conversion unit
-        const bool small_acc = g.K * (255 * 128) < (1 << 22);
         constexpr int kChunks = BN / 64;                     // 32-column chunks per warp
         int64_t staged_nt = -1;
         for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
             const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
             const int acc = local_tile & 1;
             const uint32_t acc_use = local_tile >> 1;
-            // per-column scale and bias, staged in shared memory whenever the column tile changes
-            if (need_f && nt != staged_nt) {
+            if (ev.need_f && nt != staged_nt) {              // new column tile: new scale / bias
                 staged_nt = nt;
-                epi_bar_sync();                             // previous tile's readers are done
-                for (int c = et; c < BN; c += kNumEpiWarps * 32) {
-                    const int64_t col = nt * BN + c;
-                    const bool ok = col < g.N;
-                    s_scale[c] = ok ? __ldg(g.scale + col) : 0.0f;
-                    s_bias[c] = (ok && g.bias) ? __ldg(g.bias + col) : 0.0f;
-                }
-                epi_bar_sync();
+                epi_stage_scale_bias(g, nt * BN, BN, et, s_scale, s_bias);
             }
             mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status);
             tc_fence_after();
@@ -431,65 +531,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 const int ct = cbase + ch * 32;              // column inside the tile
                 const int64_t col0 = nt * BN + ct;
                 if (!row_ok || col0 >= g.N) continue;
-                const int64_t off = row * g.N + col0;
-                const bool full = vec_ok && (col0 + 32 <= g.N);
-                if (g.acc_out) {
-                    if (full) {
-                        int4 *dst = reinterpret_cast<int4 *>(g.acc_out + off);
-#pragma unroll
-                        for (int q = 0; q < 8; ++q)
-                            dst[q] = make_int4((int)v[4 * q], (int)v[4 * q + 1], (int)v[4 * q + 2], (int)v[4 * q + 3]);
-                    } else {
-                        for (int i = 0; i < 32 && col0 + i < g.N; ++i) g.acc_out[off + i] = (int32_t)v[i];
-                    }
-                }
-                if (need_f) {
-                    // v[i] becomes the fp32 value's bits in place
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const float4 sc = *reinterpret_cast<const float4 *>(&s_scale[ct + 4 * q]);
-                        const float4 bi = *reinterpret_cast<const float4 *>(&s_bias[ct + 4 * q]);
-                        if (small_acc) {
-                            v[4 * q + 0] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 0], sc.x, bi.x, relu_op));
-                            v[4 * q + 1] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 1], sc.y, bi.y, relu_op));
-                            v[4 * q + 2] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 2], sc.z, bi.z, relu_op));
-                            v[4 * q + 3] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 3], sc.w, bi.w, relu_op));
-                        } else {
-                            v[4 * q + 0] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 0], sc.x, bi.x, relu_op));
-                            v[4 * q + 1] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 1], sc.y, bi.y, relu_op));
-                            v[4 * q + 2] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 2], sc.z, bi.z, relu_op));
-                            v[4 * q + 3] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 3], sc.w, bi.w, relu_op));
-                        }
-                    }
-                    if (g.f32_out) {
-                        if (full) {
-                            uint4 *dst = reinterpret_cast<uint4 *>(g.f32_out + off);
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) dst[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-                        } else {
-                            for (int i = 0; i < 32 && col0 + i < g.N; ++i) g.f32_out[off + i] = __uint_as_float(v[i]);
-                        }
-                    }
-                    if (g.u8_out) {
-                        uint32_t w[8];
-#pragma unroll
-                        for (int q = 0; q < 8; ++q)
-                            w[q] = pack4(requant_bits(__uint_as_float(v[4 * q]), g.inv_out_scale),
-                                         requant_bits(__uint_as_float(v[4 * q + 1]), g.inv_out_scale),
-                                         requant_bits(__uint_as_float(v[4 * q + 2]), g.inv_out_scale),
-                                         requant_bits(__uint_as_float(v[4 * q + 3]), g.inv_out_scale));
-                        if (full && u8_wide) {
-                            st_global_v8(g.u8_out + off, w);
-                        } else if (full) {
-                            uint4 *dst = reinterpret_cast<uint4 *>(g.u8_out + off);
-                            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-                        } else {
-                            for (int i = 0; i < 32 && col0 + i < g.N; ++i)
-                                g.u8_out[off + i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
-                        }
-                    }
-                }
+                epi_chunk(ev, v, row, col0, ct, s_scale, s_bias);
             }
         }
     } else if (MODE != SPARQ_MODE_NONE) {
