@@ -66,10 +66,13 @@ struct XformDev {
 
 // Mask of the bits BELOW the window for each of the four bytes of x (Section 3.1: the
 // window's top bit is the leading one, or the window sits at the bottom).  The window
-// width is WT when WT != 0, else the run-time value w_rt.  widen_c / rounds move a
-// window that landed on a disallowed placement up to the next allowed one.
-template <int WT>
-SPARQ_HD uint32_t drop_mask(uint32_t x, int w_rt, uint32_t widen_c, int rounds)
+// width is WT when WT != 0, else the run-time value w_rt.  With WIDEN, a window that landed
+// on a disallowed placement moves up to the next allowed one: one step `m |= (m << 1) & c`
+// moves every byte that sits on a disallowed shift up by one and leaves the others alone,
+// so three unconditional steps cover the longest possible run (n - 1 <= 3) and need no
+// branch.
+template <int WT, bool WIDEN>
+SPARQ_HD uint32_t drop_mask(uint32_t x, int w_rt, uint32_t widen_c)
 {
     const int w = WT ? WT : w_rt;
     const uint32_t low = 0x01010101u * (0xFFu >> w);
@@ -77,7 +80,11 @@ SPARQ_HD uint32_t drop_mask(uint32_t x, int w_rt, uint32_t widen_c, int rounds)
     m |= (m >> 1) & 0x7F7F7F7Fu;                 // smear the leading one downwards
     if (!WT || 8 - WT > 2) m |= (m >> 2) & 0x3F3F3F3Fu;
     if (!WT || 8 - WT > 4) m |= (m >> 4) & 0x0F0F0F0Fu;
-    for (int r = 0; r < rounds; ++r) m |= (m << 1) & widen_c;
+    if (WIDEN) {
+        m |= (m << 1) & widen_c;
+        m |= (m << 1) & widen_c;
+        m |= (m << 1) & widen_c;
+    }
     return m;
 }
 
@@ -99,20 +106,23 @@ SPARQ_HD uint32_t apply_mask(uint32_t x, uint32_t m, int w)
 
 // T on four packed activations (bytes 0,1 and bytes 2,3 are the pairs of Eq. 2).
 // N = 2, 3, 4 fixes the window width at compile time; N = 0 takes it from d.n.
-template <int MODE, int N, bool RND>
+// WIDEN = false is only valid for full placement sets (d.rounds == 0).
+template <int MODE, int N, bool RND, bool WIDEN>
 SPARQ_HD uint32_t xform_word(uint32_t x, const XformDev &d)
 {
     if (MODE == SPARQ_MODE_NONE) return x;
     const int n = N ? N : d.n;
-    uint32_t q = apply_mask<RND>(x, drop_mask<N>(x, n, d.widen_c, d.rounds), n);
+    uint32_t q = apply_mask<RND>(x, drop_mask<N, WIDEN>(x, n, d.widen_c), n);
     if (MODE == SPARQ_MODE_BSPARQ) return q;
     // vSPARQ: a byte whose partner is zero keeps the 2n-bit budget (all 8 bits for n = 4;
     // a 2n-bit window at any shift 0..8-2n otherwise, Section 5.1).
     uint32_t lone = x;
     if (N == 2 || N == 3) {
-        lone = apply_mask<RND>(x, drop_mask<(N == 4 ? 0 : 2 * N)>(x, 2 * n, 0u, 0), 2 * n);
-    } else if (N == 0 && 2 * n < 8) {
-        lone = apply_mask<RND>(x, drop_mask<0>(x, 2 * n, 0u, 0), 2 * n);
+        lone = apply_mask<RND>(x, drop_mask<(N == 4 ? 0 : 2 * N), false>(x, 2 * n, 0u), 2 * n);
+    } else if (N == 0) {
+        // run-time width: n = 4 gives a window of 8 bits, whose drop mask is empty
+        const int w2 = 2 * n;
+        lone = apply_mask<RND>(x, w2 < 8 ? drop_mask<0, false>(x, w2, 0u) : 0u, w2 < 8 ? w2 : 7);
     }
     uint32_t nz = ((x & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | x;   // bit 7 of each byte: byte != 0
     uint32_t partner_nz = prmt(nz, nz, 0xAB89u);           // swap within pairs, replicate bit 7

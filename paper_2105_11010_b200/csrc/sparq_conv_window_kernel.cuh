@@ -52,7 +52,7 @@ struct WindowArgs {
 
 // dynamic shared memory the kernel may ask for: 227 KB minus room for its static variables
 constexpr int kWindowMaxDynSmem = 232448 - 4096;
-constexpr int kMaxWinBufs = 3;
+constexpr int kMaxWinBufs = 4;
 constexpr int kMaxBStages = 8;
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w, int h, int n)
@@ -184,6 +184,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_i8(BN);
             uint32_t wt = 0, it = 0;
+            const uint64_t bdesc_base = make_smem_desc<CB>(b_base);
             if (B_RESIDENT) mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status);
             for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
                 const int acc = wt & 1;
@@ -196,31 +197,33 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 uint32_t first = 1;
+                int kb = 0;
                 for (int cb = 0; cb < g.c_blocks; ++cb) {
-                    const uint32_t plane = win_buf(b) + (uint32_t)cb * g.plane_bytes;
-                    for (int tap = 0; tap < taps; ++tap) {
-                        const int kb = cb * taps + tap;
-                        uint32_t bsm;
-                        int s = 0;
-                        if (B_RESIDENT) {
-                            bsm = b_slot(kb);
-                        } else {
-                            s = it % g.b_stages;
-                            mbar_wait(smem_u32(&bar_b_full[s]), (it / g.b_stages) & 1, abort_flag, g.status);
-                            tc_fence_after();
-                            bsm = b_slot(s);
-                        }
-                        const int shift_rows = (tap / g.S) * g.Wp + (tap % g.S);
-                        const uint64_t adesc = make_smem_desc<CB>(plane + (uint32_t)shift_rows * CB);
-                        const uint64_t bdesc = make_smem_desc<CB>(bsm);
+                    // descriptor of the window's channel block; a tap adds its row shift
+                    const uint64_t adesc_plane = make_smem_desc<CB>(win_buf(b) + (uint32_t)cb * g.plane_bytes);
+                    uint32_t row_shift = 0;                         // r * Wp
+                    for (int fr = 0; fr < g.R; ++fr, row_shift += (uint32_t)g.Wp) {
+                        for (int fs = 0; fs < g.S; ++fs, ++kb) {
+                            uint64_t bdesc;
+                            int s = 0;
+                            if (B_RESIDENT) {
+                                bdesc = bdesc_base + (uint64_t)((uint32_t)kb * (uint32_t)(kBBlock >> 4));
+                            } else {
+                                s = it % g.b_stages;
+                                mbar_wait(smem_u32(&bar_b_full[s]), (it / g.b_stages) & 1, abort_flag, g.status);
+                                tc_fence_after();
+                                bdesc = bdesc_base + (uint64_t)((uint32_t)s * (uint32_t)(kBBlock >> 4));
+                            }
+                            const uint64_t adesc = adesc_plane + (uint64_t)((row_shift + (uint32_t)fs) * (uint32_t)(CB >> 4));
 #pragma unroll
-                        for (int k = 0; k < CB / 32; ++k) {
-                            tc_mma_i8(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, first ? 0u : 1u);
-                            first = 0;
-                        }
-                        if (!B_RESIDENT) {
-                            tc_commit(smem_u32(&bar_b_empty[s]));
-                            ++it;
+                            for (int k = 0; k < CB / 32; ++k) {
+                                tc_mma_i8(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, first ? 0u : 1u);
+                                first = 0;
+                            }
+                            if (!B_RESIDENT) {
+                                tc_commit(smem_u32(&bar_b_empty[s]));
+                                ++it;
+                            }
                         }
                     }
                 }
@@ -282,35 +285,32 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         const int xt = threadIdx.x - kFirstXfWarp * 32;
         constexpr int kXfThreads = kNumXfWarps * 32;
         const XformDev xf = g.xf;
-        const int box_vecs = g.box_bytes / 16;
+        // whole groups of kXfThreads * 4 vectors; the tail group runs into the plane's slack
+        // rows, which no valid output reads (the host sizes the plane for it)
+        const int groups = (g.box_bytes + kXfThreads * 64 - 1) / (kXfThreads * 64);
         uint32_t wt = 0;
         for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
             const int b = wt % g.win_bufs;
             mbar_wait(smem_u32(&bar_win_full[b]), (wt / g.win_bufs) & 1, abort_flag, g.status);
             for (int cb = 0; cb < g.c_blocks; ++cb) {
-                const uint32_t plane = win_buf(b) + (uint32_t)cb * g.plane_bytes;
-                for (int v0 = xt; v0 < box_vecs; v0 += 4 * kXfThreads) {
+                const uint32_t base = win_buf(b) + (uint32_t)cb * g.plane_bytes + (uint32_t)xt * 16u;
+                for (int grp = 0; grp < groups; ++grp) {
+                    const uint32_t gbase = base + (uint32_t)grp * (kXfThreads * 64);
                     uint4 v[4];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int vi = v0 + j * kXfThreads;
-                        if (vi < box_vecs)
-                            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                                         : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w)
-                                         : "r"(plane + (uint32_t)vi * 16u));
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                     : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w)
+                                     : "r"(gbase + (uint32_t)(j * kXfThreads * 16)));
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const int vi = v0 + j * kXfThreads;
-                        if (vi < box_vecs) {
-                            v[j].x = xform_word<MODE, XN, RND>(v[j].x, xf);
-                            v[j].y = xform_word<MODE, XN, RND>(v[j].y, xf);
-                            v[j].z = xform_word<MODE, XN, RND>(v[j].z, xf);
-                            v[j].w = xform_word<MODE, XN, RND>(v[j].w, xf);
-                            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
-                                         :: "r"(plane + (uint32_t)vi * 16u),
-                                            "r"(v[j].x), "r"(v[j].y), "r"(v[j].z), "r"(v[j].w) : "memory");
-                        }
+                        v[j].x = xform_word<MODE, XN, RND, XN == 0>(v[j].x, xf);
+                        v[j].y = xform_word<MODE, XN, RND, XN == 0>(v[j].y, xf);
+                        v[j].z = xform_word<MODE, XN, RND, XN == 0>(v[j].z, xf);
+                        v[j].w = xform_word<MODE, XN, RND, XN == 0>(v[j].w, xf);
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
+                                     :: "r"(gbase + (uint32_t)(j * kXfThreads * 16)),
+                                        "r"(v[j].x), "r"(v[j].y), "r"(v[j].z), "r"(v[j].w) : "memory");
                     }
                 }
             }

@@ -112,15 +112,19 @@ static int pick_bn(int64_t M, int64_t N, int sms)
     return (N <= 64) ? 64 : best;
 }
 
+// Window-width argument of the launchers: 4 selects the kernels specialized for n = 4 with
+// all five placements; anything else (0) the general ones.
+static int variant_n(const XformArgs &x) { return (x.n == 4 && x.widen_rounds == 0) ? 4 : 0; }
+
 static cudaError_t launch(int bn, int bk, const CUtensorMap &ma, const CUtensorMap &mb, const GemmArgs &g,
                           const XformArgs &x, int grid, cudaStream_t st)
 {
-    if (bn == 64 && bk == 64) return launch_gemm_shape<64, 64>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
-    if (bn == 64) return launch_gemm_shape<64, 128>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
-    if (bn == 128 && bk == 64) return launch_gemm_shape<128, 64>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
-    if (bn == 128) return launch_gemm_shape<128, 128>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
-    if (bk == 64) return launch_gemm_shape<256, 64>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
-    return launch_gemm_shape<256, 128>(ma, mb, g, x.mode, x.n, x.rnd, grid, st);
+    if (bn == 64 && bk == 64) return launch_gemm_shape<64, 64>(ma, mb, g, x.mode, variant_n(x), x.rnd, grid, st);
+    if (bn == 64) return launch_gemm_shape<64, 128>(ma, mb, g, x.mode, variant_n(x), x.rnd, grid, st);
+    if (bn == 128 && bk == 64) return launch_gemm_shape<128, 64>(ma, mb, g, x.mode, variant_n(x), x.rnd, grid, st);
+    if (bn == 128) return launch_gemm_shape<128, 128>(ma, mb, g, x.mode, variant_n(x), x.rnd, grid, st);
+    if (bk == 64) return launch_gemm_shape<256, 64>(ma, mb, g, x.mode, variant_n(x), x.rnd, grid, st);
+    return launch_gemm_shape<256, 128>(ma, mb, g, x.mode, variant_n(x), x.rnd, grid, st);
 }
 
 static void fill_common(GemmArgs *g, const XformArgs &x, const sparq_epilogue *e, unsigned int *status)
@@ -208,7 +212,11 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     const int taps = r * s;
     const int kb_count = taps * c_blocks;
     const int rows_alloc = (r - 1) * wp + (s - 1) + 128;
-    const int plane_bytes = (rows_alloc * cb + 1023) / 1024 * 1024;
+    // a plane holds every row the MMA may touch and the whole 16 KB groups the transform rewrites
+    const int box_bytes = cb * wp * (tr + r - 1);
+    int plane_bytes = rows_alloc * cb;
+    if (plane_bytes < (box_bytes + 16383) / 16384 * 16384) plane_bytes = (box_bytes + 16383) / 16384 * 16384;
+    plane_bytes = (plane_bytes + 1023) / 1024 * 1024;
     const int win_bytes = plane_bytes * c_blocks;
     const int tiles_per_img = (ho + tr - 1) / tr;
     const int64_t m_tiles = (int64_t)n * tiles_per_img;
@@ -228,13 +236,19 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     if (bn != 256 && n_tiles == 1 && 1024 + 2 * win_bytes + kb_count * b_block <= kMaxDynSmem) {
         resident = true;
         b_stages = kb_count;
-        if (1024 + 3 * win_bytes + kb_count * b_block <= kMaxDynSmem) win_bufs = 3;
+        while (win_bufs < kMaxWinBufs && 1024 + (win_bufs + 1) * win_bytes + kb_count * b_block <= kMaxDynSmem) ++win_bufs;
     } else {
         if (bn == 64) return 0;                          // only the resident form is built for 64-wide tiles
         const int left = kMaxDynSmem - 1024 - 2 * win_bytes;
         b_stages = left / b_block;
         if (b_stages > kMaxBStages) b_stages = kMaxBStages;
         if (b_stages < 2) return 0;
+        // spare room beyond four weight stages goes to a third window buffer
+        if (b_stages > 4 && 1024 + 3 * win_bytes + 4 * b_block <= kMaxDynSmem) {
+            win_bufs = 3;
+            b_stages = (kMaxDynSmem - 1024 - 3 * win_bytes) / b_block;
+            if (b_stages > kMaxBStages) b_stages = kMaxBStages;
+        }
     }
     const int smem_bytes = 1024 + win_bufs * win_bytes + b_stages * b_block;
 
@@ -250,7 +264,7 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     g.N = cout; g.K = K;
     g.n_img = n; g.H = h; g.W = w; g.C = c; g.R = r; g.S = s; g.pad_h = pad_h; g.pad_w = pad_w; g.Ho = ho; g.Wo = wo;
     g.Wp = wp; g.TR = tr; g.tiles_per_img = tiles_per_img; g.c_blocks = c_blocks;
-    g.box_bytes = cb * wp * (tr + r - 1);
+    g.box_bytes = box_bytes;
     g.plane_bytes = plane_bytes;
     g.win_bufs = win_bufs;
     g.b_stages = b_stages;
@@ -261,10 +275,10 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     const int64_t tiles = m_tiles * n_tiles;
     const int grid = (int)(tiles < sms ? tiles : sms);
     cudaError_t ce;
-    if (bn == 64) ce = launch_window_shape<64, 64, true>(mx, mw, g, x.mode, x.n, x.rnd, grid, smem_bytes, st);
-    else if (bn == 128 && resident) ce = launch_window_shape<128, 128, true>(mx, mw, g, x.mode, x.n, x.rnd, grid, smem_bytes, st);
-    else if (bn == 128) ce = launch_window_shape<128, 128, false>(mx, mw, g, x.mode, x.n, x.rnd, grid, smem_bytes, st);
-    else ce = launch_window_shape<256, 128, false>(mx, mw, g, x.mode, x.n, x.rnd, grid, smem_bytes, st);
+    if (bn == 64) ce = launch_window_shape<64, 64, true>(mx, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
+    else if (bn == 128 && resident) ce = launch_window_shape<128, 128, true>(mx, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
+    else if (bn == 128) ce = launch_window_shape<128, 128, false>(mx, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
+    else ce = launch_window_shape<256, 128, false>(mx, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
     if (ce != cudaSuccess) return cuda_error(ce, "sparq_conv_window_kernel launch");
     return 1;
 }

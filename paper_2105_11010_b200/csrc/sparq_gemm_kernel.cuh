@@ -556,10 +556,10 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                                  : "r"(base + (uint32_t)(j * kXfThreads * 16)));
 #pragma unroll
                 for (int j = 0; j < kPerThread; ++j) {
-                    v[j].x = xform_word<MODE, XN, RND>(v[j].x, xf);
-                    v[j].y = xform_word<MODE, XN, RND>(v[j].y, xf);
-                    v[j].z = xform_word<MODE, XN, RND>(v[j].z, xf);
-                    v[j].w = xform_word<MODE, XN, RND>(v[j].w, xf);
+                    v[j].x = xform_word<MODE, XN, RND, XN == 0>(v[j].x, xf);
+                    v[j].y = xform_word<MODE, XN, RND, XN == 0>(v[j].y, xf);
+                    v[j].z = xform_word<MODE, XN, RND, XN == 0>(v[j].z, xf);
+                    v[j].w = xform_word<MODE, XN, RND, XN == 0>(v[j].w, xf);
                     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
                                  :: "r"(base + (uint32_t)(j * kXfThreads * 16)),
                                     "r"(v[j].x), "r"(v[j].y), "r"(v[j].z), "r"(v[j].w) : "memory");

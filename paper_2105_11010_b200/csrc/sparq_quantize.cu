@@ -29,7 +29,7 @@ __device__ __forceinline__ void st_stream(uint4 *p, uint4 v)
                  :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-template <int MODE, int N, bool RND>
+template <int MODE, int N, bool RND, bool WIDEN>
 __global__ void __launch_bounds__(kThreads)
 quantize_vec_kernel(const uint4 *in, uint4 *out, size_t nvec, XformDev d)
 {
@@ -46,10 +46,10 @@ quantize_vec_kernel(const uint4 *in, uint4 *out, size_t nvec, XformDev d)
         for (int j = 0; j < kVec; ++j) {
             if (idx[j] < nvec) {
                 uint4 o;
-                o.x = xform_word<MODE, N, RND>(v[j].x, d);
-                o.y = xform_word<MODE, N, RND>(v[j].y, d);
-                o.z = xform_word<MODE, N, RND>(v[j].z, d);
-                o.w = xform_word<MODE, N, RND>(v[j].w, d);
+                o.x = xform_word<MODE, N, RND, WIDEN>(v[j].x, d);
+                o.y = xform_word<MODE, N, RND, WIDEN>(v[j].y, d);
+                o.z = xform_word<MODE, N, RND, WIDEN>(v[j].z, d);
+                o.w = xform_word<MODE, N, RND, WIDEN>(v[j].w, d);
                 st_stream(out + idx[j], o);
             }
         }
@@ -108,10 +108,11 @@ static cudaError_t launch_vec(const uint4 *in, uint4 *out, size_t nvec, const Xf
                               int blocks, cudaStream_t st)
 {
     XformDev d{a.widen_c, a.widen_rounds, a.n};
-    if (a.rnd)
-        quantize_vec_kernel<MODE, N, true><<<blocks, kThreads, 0, st>>>(in, out, nvec, d);
-    else
-        quantize_vec_kernel<MODE, N, false><<<blocks, kThreads, 0, st>>>(in, out, nvec, d);
+    const bool widen = a.widen_rounds > 0;   // restricted placement set
+    if (a.rnd && widen) quantize_vec_kernel<MODE, N, true, true><<<blocks, kThreads, 0, st>>>(in, out, nvec, d);
+    else if (a.rnd) quantize_vec_kernel<MODE, N, true, false><<<blocks, kThreads, 0, st>>>(in, out, nvec, d);
+    else if (widen) quantize_vec_kernel<MODE, N, false, true><<<blocks, kThreads, 0, st>>>(in, out, nvec, d);
+    else quantize_vec_kernel<MODE, N, false, false><<<blocks, kThreads, 0, st>>>(in, out, nvec, d);
     return cudaGetLastError();
 }
 
