@@ -54,6 +54,7 @@ struct WindowArgs {
 constexpr int kWindowMaxDynSmem = 232448 - 4096;
 constexpr int kMaxWinBufs = 4;
 constexpr int kMaxBStages = 8;
+constexpr int kMaxKb = 128;     // (tap, channel block) pairs the MMA warp keeps a table for
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w, int h, int n)
 {
@@ -74,12 +75,16 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
     __shared__ uint32_t tmem_base_slot;
     __shared__ uint32_t abort_word;
     __shared__ __align__(16) float s_scale[BN], s_bias[BN];
+    // per (channel block, tap): .x = offset of the tap's A rows inside a window buffer,
+    // .y = offset of the resident weight block; both in 16-byte units (descriptor units)
+    __shared__ uint2 s_tab[kMaxKb];
 
     constexpr int kBBlock = BN * CB;                   // one (tap, channel block) of weights
     constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     volatile uint32_t *abort_flag = &abort_word;
+    const long long cta_t0 = SPARQ_PROF_NOW();
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t win_bytes = (uint32_t)g.plane_bytes * (uint32_t)g.c_blocks;
@@ -109,6 +114,12 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
+        for (int kb = lane; kb < kb_count; kb += 32) {
+            const int cb = kb / taps, tap = kb % taps;
+            const uint32_t rows = (uint32_t)((tap / g.S) * g.Wp + (tap % g.S));
+            s_tab[kb] = make_uint2(((uint32_t)cb * (uint32_t)g.plane_bytes + rows * CB) >> 4,
+                                   (uint32_t)kb * (uint32_t)(kBBlock >> 4));
+        }
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      :: "r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -137,13 +148,15 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             }
             uint32_t wt = 0;      // window counter
             uint32_t it = 0;      // streamed weight-block counter
+            long long pw = 0;
+            const long long pt0 = SPARQ_PROF_NOW();
             for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
                 const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
                 const int img = (int)(mt / g.tiles_per_img);
                 const int oh0 = (int)(mt % g.tiles_per_img) * g.TR;
                 const int b = wt % g.win_bufs;
                 const uint32_t use = wt / g.win_bufs;
-                if (use > 0) mbar_wait(smem_u32(&bar_win_empty[b]), (use - 1) & 1, abort_flag, g.status);
+                if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_win_empty[b]), (use - 1) & 1, abort_flag, g.status));
                 if (*abort_flag) break;
                 const uint32_t wfull = smem_u32(&bar_win_full[b]);
                 mbar_expect_tx(wfull, (uint32_t)g.box_bytes * (uint32_t)g.c_blocks);
@@ -164,6 +177,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 }
                 if (*abort_flag) break;
             }
+            SPARQ_PROF_STORE(0, pw);
+            SPARQ_PROF_STORE(1, SPARQ_PROF_NOW() - pt0);
             if (*abort_flag) {
                 // wait (bounded) for copies still in flight so that none lands after exit
                 const uint32_t wfirst = wt > (uint32_t)g.win_bufs ? wt - g.win_bufs : 0;
@@ -183,53 +198,56 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         // ================= MMA issuer =================
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_i8(BN);
-            uint32_t wt = 0, it = 0;
-            const uint64_t bdesc_base = make_smem_desc<CB>(b_base);
-            if (B_RESIDENT) mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status);
+            const uint64_t desc0 = make_smem_desc<CB>(smem_base);
+            const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
+            const uint32_t win_lo0 = (uint32_t)desc0;
+            const uint32_t b_lo0 = win_lo0 + (((uint32_t)g.win_bufs * win_bytes) >> 4);
+            uint32_t wt = 0;
+            int b = 0;  uint32_t wph = 0;      // window buffer and its phase parity
+            int s = 0;  uint32_t bph = 0;      // streamed weight stage and its phase parity
+            long long mw = 0, ma = 0, mb = 0, mi = 0;
+            const long long mt0 = SPARQ_PROF_NOW();
+            if (B_RESIDENT) SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status));
             for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
                 const int acc = wt & 1;
                 const uint32_t acc_use = wt >> 1;
-                if (acc_use > 0) mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status);
-                const int b = wt % g.win_bufs;
-                const uint32_t wph = (wt / g.win_bufs) & 1;
-                if (MODE == SPARQ_MODE_NONE) mbar_wait(smem_u32(&bar_win_full[b]), wph, abort_flag, g.status);
-                else mbar_wait(smem_u32(&bar_win_xf[b]), wph, abort_flag, g.status);
+                if (acc_use > 0) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status));
+                if (MODE == SPARQ_MODE_NONE) SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_full[b]), wph, abort_flag, g.status));
+                else SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b]), wph, abort_flag, g.status));
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                uint32_t first = 1;
-                int kb = 0;
-                for (int cb = 0; cb < g.c_blocks; ++cb) {
-                    // descriptor of the window's channel block; a tap adds its row shift
-                    const uint64_t adesc_plane = make_smem_desc<CB>(win_buf(b) + (uint32_t)cb * g.plane_bytes);
-                    uint32_t row_shift = 0;                         // r * Wp
-                    for (int fr = 0; fr < g.R; ++fr, row_shift += (uint32_t)g.Wp) {
-                        for (int fs = 0; fs < g.S; ++fs, ++kb) {
-                            uint64_t bdesc;
-                            int s = 0;
-                            if (B_RESIDENT) {
-                                bdesc = bdesc_base + (uint64_t)((uint32_t)kb * (uint32_t)(kBBlock >> 4));
-                            } else {
-                                s = it % g.b_stages;
-                                mbar_wait(smem_u32(&bar_b_full[s]), (it / g.b_stages) & 1, abort_flag, g.status);
-                                tc_fence_after();
-                                bdesc = bdesc_base + (uint64_t)((uint32_t)s * (uint32_t)(kBBlock >> 4));
-                            }
-                            const uint64_t adesc = adesc_plane + (uint64_t)((row_shift + (uint32_t)fs) * (uint32_t)(CB >> 4));
+                const uint32_t a_lo0 = win_lo0 + (uint32_t)b * (win_bytes >> 4);
+                const long long is0 = SPARQ_PROF_NOW();
+                for (int kb = 0; kb < kb_count; ++kb) {
+                    const uint2 e = s_tab[kb];
+                    uint32_t b_lo;
+                    if (B_RESIDENT) {
+                        b_lo = b_lo0 + e.y;
+                    } else {
+                        SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status));
+                        tc_fence_after();
+                        b_lo = b_lo0 + (uint32_t)s * (uint32_t)(kBBlock >> 4);
+                    }
+                    const uint32_t a_lo = a_lo0 + e.x;
 #pragma unroll
-                            for (int k = 0; k < CB / 32; ++k) {
-                                tc_mma_i8(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, first ? 0u : 1u);
-                                first = 0;
-                            }
-                            if (!B_RESIDENT) {
-                                tc_commit(smem_u32(&bar_b_empty[s]));
-                                ++it;
-                            }
-                        }
+                    for (int k = 0; k < CB / 32; ++k)
+                        tc_mma_i8_parts(d_tmem, desc_hi, a_lo + (uint32_t)(k * 2), b_lo + (uint32_t)(k * 2), idesc,
+                                        (kb > 0 || k > 0) ? 1u : 0u);
+                    if (!B_RESIDENT) {
+                        tc_commit(smem_u32(&bar_b_empty[s]));
+                        if (++s == g.b_stages) { s = 0; bph ^= 1u; }
                     }
                 }
+                mi += SPARQ_PROF_NOW() - is0;
                 tc_commit(smem_u32(&bar_win_empty[b]));       // window reusable once these MMAs retire
                 tc_commit(smem_u32(&bar_acc_full[acc]));      // accumulator complete
+                if (++b == g.win_bufs) { b = 0; wph ^= 1u; }
             }
+            SPARQ_PROF_STORE(2, mw);
+            SPARQ_PROF_STORE(3, ma);
+            SPARQ_PROF_STORE(11, mb);
+            SPARQ_PROF_STORE(12, mi);
+            SPARQ_PROF_STORE(4, SPARQ_PROF_NOW() - mt0);
             tc_commit(smem_u32(&bar_done));
             mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, true);
         }
@@ -248,6 +266,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         const int tr = slot / g.Wp;
         const int ow = slot - tr * g.Wp;
         const bool slot_ok = (tr < g.TR) && (ow < g.Wo);
+        long long ew = 0;
+        const long long et0 = SPARQ_PROF_NOW();
         for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
             const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
             const int acc = wt & 1;
@@ -256,7 +276,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 staged_nt = nt;
                 epi_stage_scale_bias(g, nt * BN, BN, et, s_scale, s_bias);
             }
-            mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status);
+            SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status));
             tc_fence_after();
             const int img = (int)(mt / g.tiles_per_img);
             const int oh = (int)(mt % g.tiles_per_img) * g.TR + tr;
@@ -280,6 +300,10 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 epi_chunk(ev, v, row, col0, ct, s_scale, s_bias);
             }
         }
+        if (warp == kFirstEpiWarp && lane == 0) {
+            SPARQ_PROF_STORE(5, ew);
+            SPARQ_PROF_STORE(6, SPARQ_PROF_NOW() - et0);
+        }
     } else if (MODE != SPARQ_MODE_NONE) {
         // ================= transform: once per window =================
         const int xt = threadIdx.x - kFirstXfWarp * 32;
@@ -289,9 +313,11 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         // rows, which no valid output reads (the host sizes the plane for it)
         const int groups = (g.box_bytes + kXfThreads * 64 - 1) / (kXfThreads * 64);
         uint32_t wt = 0;
+        long long xw = 0;
+        const long long xt0 = SPARQ_PROF_NOW();
         for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
             const int b = wt % g.win_bufs;
-            mbar_wait(smem_u32(&bar_win_full[b]), (wt / g.win_bufs) & 1, abort_flag, g.status);
+            SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_win_full[b]), (wt / g.win_bufs) & 1, abort_flag, g.status));
             for (int cb = 0; cb < g.c_blocks; ++cb) {
                 const uint32_t base = win_buf(b) + (uint32_t)cb * g.plane_bytes + (uint32_t)xt * 16u;
                 for (int grp = 0; grp < groups; ++grp) {
@@ -318,10 +344,15 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bar_win_xf[b]));
         }
+        if (warp == kFirstXfWarp && lane == 0) {
+            SPARQ_PROF_STORE(7, xw);
+            SPARQ_PROF_STORE(8, SPARQ_PROF_NOW() - xt0);
+        }
     }
 
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) SPARQ_PROF_STORE(10, SPARQ_PROF_NOW() - cta_t0);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"

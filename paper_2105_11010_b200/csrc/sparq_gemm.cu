@@ -8,6 +8,10 @@
 
 namespace sparq {
 
+#ifdef SPARQ_PROF
+__device__ long long g_prof[148 * 16];
+#endif
+
 void release_gemm_state() {}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -211,6 +215,7 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     const int c_blocks = c / cb;
     const int taps = r * s;
     const int kb_count = taps * c_blocks;
+    if (kb_count > kMaxKb) return 0;
     const int rows_alloc = (r - 1) * wp + (s - 1) + 128;
     // a plane holds every row the MMA may touch and the whole 16 KB groups the transform rewrites
     const int box_bytes = cb * wp * (tr + r - 1);
@@ -402,3 +407,11 @@ extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, in
     if (ce != cudaSuccess) return cuda_error(ce, "sparq_gemm_kernel (convolution) launch");
     return SPARQ_OK;
 }
+
+#ifdef SPARQ_PROF
+// Profiling builds only: copies the per-CTA role counters of the last fused launch.
+extern "C" __attribute__((visibility("default"))) int sparq_prof_read(long long *out)
+{
+    return (int)cudaMemcpyFromSymbol(out, sparq::g_prof, sizeof(long long) * 148 * 16);
+}
+#endif

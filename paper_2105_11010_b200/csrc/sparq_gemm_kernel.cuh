@@ -39,6 +39,21 @@ constexpr int kGemmThreads = 32 * (kFirstXfWarp + kNumXfWarps);
 constexpr int kSmemBudget = 200 * 1024;  // for the stage ring
 constexpr long long kWaitLimitCycles = 2000000000LL;
 
+// Optional per-role cycle counters (builds with -DSPARQ_PROF only): how long each warp role
+// waited on its barriers and how long it ran, per CTA.  Compiled out otherwise.
+#ifdef SPARQ_PROF
+extern __device__ long long g_prof[148 * 16];
+#define SPARQ_PROF_NOW() clock64()
+#define SPARQ_PROF_STORE(slot, v) (g_prof[blockIdx.x * 16 + (slot)] = (v))
+#else
+#define SPARQ_PROF_NOW() 0LL
+#define SPARQ_PROF_STORE(slot, v) ((void)(v))
+#endif
+#define SPARQ_PROF_WAIT(accum, stmt) do { const long long t_ = SPARQ_PROF_NOW(); stmt; accum += SPARQ_PROF_NOW() - t_; } while (0)
+// slots: 0 producer wait, 1 producer total, 2 MMA wait for operands, 3 MMA wait for a free
+// accumulator, 4 MMA total, 5 epilogue wait, 6 epilogue total, 7 transform wait,
+// 8 transform total, 10 CTA total, 11 MMA wait for weights, 12 MMA issue section
+
 struct GemmArgs {
     // problem
     int64_t M, N, K;        // GEMM view (K = r*s*c for the convolution)
@@ -156,6 +171,21 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint6
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
         :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// Same, with both descriptors given as (shared high word, low word): the high words of two
+// descriptors with the same row length and swizzle are equal, and the issuing thread then
+// only does 32-bit arithmetic per instruction.
+__device__ __forceinline__ void tc_mma_i8_parts(uint32_t d_tmem, uint32_t desc_hi, uint32_t a_lo, uint32_t b_lo,
+                                                uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t}"
+        :: "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 
 // Shared-memory matrix descriptor of a K-major tile whose rows are ROW_BYTES long
@@ -385,6 +415,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     volatile uint32_t *abort_flag = &abort_word;
+    const long long cta_t0 = SPARQ_PROF_NOW();
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     auto a_stage = [&](int s) { return smem_base + (uint32_t)s * Cfg::kStageBytes; };
@@ -423,6 +454,8 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         // ================= TMA producer =================
         if (lane == 0) {
             uint32_t it = 0;   // running stage counter across tiles
+            long long pw = 0;
+            const long long pt0 = SPARQ_PROF_NOW();
             for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
                 const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
                 const int64_t m0 = mt * kBM;
@@ -438,7 +471,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 for (int kb = 0; kb < kb_count; ++kb, ++it) {
                     const int s = it % S;
                     const uint32_t use = it / S;
-                    if (use > 0) mbar_wait(smem_u32(&bar_empty[s]), (use - 1) & 1, abort_flag, g.status);
+                    if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_empty[s]), (use - 1) & 1, abort_flag, g.status));
                     if (*abort_flag) break;   // stop issuing copies once the CTA has given up
                     const uint32_t full = smem_u32(&bar_full[s]);
                     mbar_expect_tx(full, Cfg::kStageBytes);
@@ -453,6 +486,8 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 }
                 if (*abort_flag) break;
             }
+            SPARQ_PROF_STORE(0, pw);
+            SPARQ_PROF_STORE(1, SPARQ_PROF_NOW() - pt0);
             // After an abort: wait (bounded) for the copies this thread still has in
             // flight, so that none lands after the CTA has exited.
             if (*abort_flag) {
@@ -466,29 +501,38 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         // ================= MMA issuer =================
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_i8(BN);
-            uint32_t it = 0, local_tile = 0;
+            const uint64_t desc0 = make_smem_desc<BK>(smem_base);
+            const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
+            const uint32_t a_lo0 = (uint32_t)desc0;
+            const uint32_t b_lo0 = a_lo0 + (uint32_t)(Cfg::kABytes >> 4);
+            uint32_t local_tile = 0;
+            int s = 0;             // stage
+            uint32_t ph = 0;       // its phase parity
+            long long mw = 0, ma = 0;
+            const long long mt0 = SPARQ_PROF_NOW();
             for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
                 const int acc = local_tile & 1;
                 const uint32_t acc_use = local_tile >> 1;
-                if (acc_use > 0) mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status);
+                if (acc_use > 0) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status));
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                for (int kb = 0; kb < kb_count; ++kb, ++it) {
-                    const int s = it % S;
-                    const uint32_t ph = (it / S) & 1;
-                    if (MODE == SPARQ_MODE_NONE) mbar_wait(smem_u32(&bar_full[s]), ph, abort_flag, g.status);
-                    else mbar_wait(smem_u32(&bar_xf[s]), ph, abort_flag, g.status);
+                for (int kb = 0; kb < kb_count; ++kb) {
+                    if (MODE == SPARQ_MODE_NONE) SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_full[s]), ph, abort_flag, g.status));
+                    else SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_xf[s]), ph, abort_flag, g.status));
                     tc_fence_after();
-                    const uint64_t adesc = make_smem_desc<BK>(a_stage(s));
-                    const uint64_t bdesc = make_smem_desc<BK>(b_stage(s));
+                    const uint32_t st_off = (uint32_t)s * (uint32_t)(Cfg::kStageBytes >> 4);
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)
-                        tc_mma_i8(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
-                                  (kb > 0 || k > 0) ? 1u : 0u);
+                        tc_mma_i8_parts(d_tmem, desc_hi, a_lo0 + st_off + (uint32_t)(k * 2), b_lo0 + st_off + (uint32_t)(k * 2),
+                                        idesc, (kb > 0 || k > 0) ? 1u : 0u);
                     tc_commit(smem_u32(&bar_empty[s]));       // stage reusable once these MMAs retire
+                    if (++s == S) { s = 0; ph ^= 1u; }
                 }
                 tc_commit(smem_u32(&bar_acc_full[acc]));      // accumulator complete
             }
+            SPARQ_PROF_STORE(2, mw);
+            SPARQ_PROF_STORE(3, ma);
+            SPARQ_PROF_STORE(4, SPARQ_PROF_NOW() - mt0);
             // all tensor-core work of this CTA has retired before tensor memory is freed
             tc_commit(smem_u32(&bar_done));
             mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, true);
@@ -503,6 +547,8 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         uint32_t local_tile = 0;
         constexpr int kChunks = BN / 64;                     // 32-column chunks per warp
         int64_t staged_nt = -1;
+        long long ew = 0;
+        const long long et0 = SPARQ_PROF_NOW();
         for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
             const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
             const int acc = local_tile & 1;
@@ -511,7 +557,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 staged_nt = nt;
                 epi_stage_scale_bias(g, nt * BN, BN, et, s_scale, s_bias);
             }
-            mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status);
+            SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status));
             tc_fence_after();
             const int64_t row = mt * kBM + quarter * 32 + lane;
             const bool row_ok = row < g.M;
@@ -534,6 +580,10 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 epi_chunk(ev, v, row, col0, ct, s_scale, s_bias);
             }
         }
+        if (warp == kFirstEpiWarp && lane == 0) {
+            SPARQ_PROF_STORE(5, ew);
+            SPARQ_PROF_STORE(6, SPARQ_PROF_NOW() - et0);
+        }
     } else if (MODE != SPARQ_MODE_NONE) {
         // ================= transform =================
         const int xt = threadIdx.x - kFirstXfWarp * 32;            // 0 .. 255 among the transform threads
@@ -543,10 +593,12 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         static_assert(kVecs % kXfThreads == 0, "A stage must split evenly over the transform threads");
         const XformDev xf = g.xf;
         uint32_t it = 0;
+        long long xw = 0;
+        const long long xt0 = SPARQ_PROF_NOW();
         for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < kb_count; ++kb, ++it) {
                 const int s = it % S;
-                mbar_wait(smem_u32(&bar_full[s]), (it / S) & 1, abort_flag, g.status);
+                SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_full[s]), (it / S) & 1, abort_flag, g.status));
                 const uint32_t base = a_stage(s) + (uint32_t)xt * 16u;
                 uint4 v[kPerThread];
 #pragma unroll
@@ -569,10 +621,15 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (lane == 0) mbar_arrive(smem_u32(&bar_xf[s]));
             }
         }
+        if (warp == kFirstXfWarp && lane == 0) {
+            SPARQ_PROF_STORE(7, xw);
+            SPARQ_PROF_STORE(8, SPARQ_PROF_NOW() - xt0);
+        }
     }
 
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) SPARQ_PROF_STORE(10, SPARQ_PROF_NOW() - cta_t0);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
