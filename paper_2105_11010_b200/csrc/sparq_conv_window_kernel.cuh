@@ -207,6 +207,10 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             int s = 0;  uint32_t bph = 0;      // streamed weight stage and its phase parity
             long long mw = 0, ma = 0, mb = 0, mi = 0;
             const long long mt0 = SPARQ_PROF_NOW();
+            constexpr int kRegTab = 18;         // 3x3 taps of up to two channel blocks
+            uint2 rtab[kRegTab];
+#pragma unroll
+            for (int kb = 0; kb < kRegTab; ++kb) rtab[kb] = (kb < kb_count) ? s_tab[kb] : make_uint2(0u, 0u);
             if (B_RESIDENT) SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status));
             for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
                 const int acc = wt & 1;
@@ -218,8 +222,9 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 const uint32_t a_lo0 = win_lo0 + (uint32_t)b * (win_bytes >> 4);
                 const long long is0 = SPARQ_PROF_NOW();
-                for (int kb = 0; kb < kb_count; ++kb) {
-                    const uint2 e = s_tab[kb];
+                // One (tap, channel block) of the tile: wait for its weights when they are
+                // streamed, then CB / 32 MMAs.
+                auto issue_block = [&](int kb, const uint2 e) {
                     uint32_t b_lo;
                     if (B_RESIDENT) {
                         b_lo = b_lo0 + e.y;
@@ -237,6 +242,14 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                         tc_commit(smem_u32(&bar_b_empty[s]));
                         if (++s == g.b_stages) { s = 0; bph ^= 1u; }
                     }
+                };
+                if (kb_count <= kRegTab) {
+                    // table in registers: nothing but two adds stands between consecutive MMAs
+#pragma unroll
+                    for (int kb = 0; kb < kRegTab; ++kb)
+                        if (kb < kb_count) issue_block(kb, rtab[kb]);
+                } else {
+                    for (int kb = 0; kb < kb_count; ++kb) issue_block(kb, s_tab[kb]);
                 }
                 mi += SPARQ_PROF_NOW() - is0;
                 tc_commit(smem_u32(&bar_win_empty[b]));       // window reusable once these MMAs retire
