@@ -96,6 +96,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
     const int kb_count = taps * g.c_blocks;            // weight blocks per tile
 
     if (threadIdx.x == 0) {
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_w);
         for (int b = 0; b < kMaxWinBufs; ++b) {
             mbar_init(smem_u32(&bar_win_full[b]), 1);
             mbar_init(smem_u32(&bar_win_xf[b]), kNumXfWarps);
@@ -128,6 +130,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    dep_launch();
+    dep_wait();
 
     // With resident weights there is one column tile (host guarantees N <= BN).
     const int64_t n_tiles = (g.N + BN - 1) / BN;
@@ -390,8 +394,7 @@ cudaError_t launch_window_shape(const CUtensorMap &mx, const CUtensorMap &mw, co
             if (e_ != cudaSuccess) return e_;                                                          \
             if (dev_ >= 0 && dev_ < 64) attr_set[dev_] = true;                                         \
         }                                                                                              \
-        kfn<<<grid, kGemmThreads, smem_bytes, st>>>(mx, mw, g);                                        \
-        return cudaGetLastError();                                                                     \
+        return launch_pdl(kfn, grid, smem_bytes, st, mx, mw, g);                                       \
     } while (0)
 
 #define SPARQ_DEFINE_WINDOW_SHAPE(BN_, CB_, RES_)                                                      \

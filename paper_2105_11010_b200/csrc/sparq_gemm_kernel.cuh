@@ -149,6 +149,18 @@ __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorM
         :: "r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(woff), "h"(hoff) : "memory");
 }
 
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" :: "l"(map) : "memory");
+}
+
+// Programmatic dependent launch: the kernel may start while the previous kernel on the
+// stream is still draining.  dep_launch() lets the next kernel start its own prologue;
+// dep_wait() blocks until every earlier kernel has completed and its writes are visible,
+// and is executed by every thread before it touches global memory.
+__device__ __forceinline__ void dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void fence_proxy_async_smem()
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -422,6 +434,8 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     auto b_stage = [&](int s) { return smem_base + (uint32_t)s * Cfg::kStageBytes + Cfg::kABytes; };
 
     if (threadIdx.x == 0) {
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
         for (int s = 0; s < S; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
             mbar_init(smem_u32(&bar_xf[s]), kNumXfWarps);
@@ -444,6 +458,8 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    dep_launch();
+    dep_wait();
 
     const int64_t m_tiles = (g.M + kBM - 1) / kBM;
     const int64_t n_tiles = (g.N + BN - 1) / BN;
@@ -637,6 +653,24 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     }
 }
 
+// Launch with programmatic stream serialization allowed (see dep_wait / dep_launch).
+template <class Kernel, class Args>
+cudaError_t launch_pdl(Kernel kfn, int grid, int smem_bytes, cudaStream_t st, const CUtensorMap &m0,
+                       const CUtensorMap &m1, const Args &g)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kfn, m0, m1, g);
+}
+
 // Host launcher for one tile shape; picks the transform variant.  Defined once per
 // (BN, BK) in its own translation unit.
 template <int BN, int BK>
@@ -656,8 +690,7 @@ cudaError_t launch_gemm_shape(const CUtensorMap &ma, const CUtensorMap &mb, cons
             if (e_ != cudaSuccess) return e_;                                                          \
             if (dev_ >= 0 && dev_ < 64) attr_set[dev_] = true;                                         \
         }                                                                                              \
-        kfn<<<grid, kGemmThreads, TileCfg<BN, BK>::kSmemBytes, st>>>(ma, mb, g);                       \
-        return cudaGetLastError();                                                                     \
+        return launch_pdl(kfn, grid, TileCfg<BN, BK>::kSmemBytes, st, ma, mb, g);                      \
     } while (0)
 
 #define SPARQ_DEFINE_GEMM_SHAPE(BN_, BK_)                                                              \
