@@ -100,20 +100,34 @@ static int check_epilogue(const sparq_epilogue *e)
     return SPARQ_OK;
 }
 
-static int pick_bn(int64_t M, int64_t N, int sms)
+// Tile width for the 128 x BN kernel.  Per reduction step (128 bytes of K) a CTA needs about
+//   max( transform of the A stage  ~1250 cycles when a SPARQ mode is on,
+//        MMA                       2 * BN cycles,
+//        operand fetch from L2     ~4.4 cycles per 128-byte row of A and B )
+// and the kernel takes ceil(tiles / SMs) such passes; narrow tiles add CTAs but re-fetch
+// and re-transform A once per column tile.  Pick the width with the lowest estimate.
+static int pick_bn(int64_t M, int64_t N, int sms, bool transform)
 {
     const int cand[3] = {256, 128, 64};
     const int64_t m_tiles = (M + kBM - 1) / kBM;
     int best = 64;
+    double best_cost = 0.0;
     for (int i = 0; i < 3; ++i) {
         const int bn = cand[i];
         if (bn > 64 && N <= bn / 2) continue;          // would be mostly padding
         const int64_t tiles = m_tiles * ((N + bn - 1) / bn);
-        if (tiles >= sms) return bn;                    // the widest tile that still fills the GPU
-        best = bn;
+        const int64_t rounds = (tiles + sms - 1) / sms;
+        double step = 2.0 * bn;
+        const double fetch = 4.4 * (kBM + bn);
+        if (fetch > step) step = fetch;
+        if (transform && step < 1250.0) step = 1250.0;
+        const double cost = (double)rounds * (step + 150.0);   // + fixed per-step hand-off cost
+        if (best_cost == 0.0 || cost < best_cost) {
+            best_cost = cost;
+            best = bn;
+        }
     }
-    // nothing fills the GPU: the narrowest admissible tile gives the most CTAs
-    return (N <= 64) ? 64 : best;
+    return best;
 }
 
 // Window-width argument of the launchers: 4 selects the kernels specialized for n = 4 with
@@ -157,7 +171,7 @@ static int gemm_impl(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     // reduction step: the one that pads K the least; ties go to the wider step
     const int64_t pad128 = (K + 127) / 128 * 128, pad64 = (K + 63) / 64 * 64;
     const int bk = (pad64 < pad128) ? 64 : 128;
-    const int bn = pick_bn(M, N, sms);
+    const int bn = pick_bn(M, N, sms, x.mode != SPARQ_MODE_NONE);
 
     CUtensorMap ma, mb;
     rc = encode_2d(&ma, A, K, M, lda, bk, kBM);
@@ -298,7 +312,7 @@ int gemm_with_status(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     if (rc != SPARQ_OK) return rc;
     const int64_t pad128 = (K + 127) / 128 * 128, pad64 = (K + 63) / 64 * 64;
     const int bk = (pad64 < pad128) ? 64 : 128;
-    const int bn = pick_bn(M, N, sms);
+    const int bn = pick_bn(M, N, sms, x.mode != SPARQ_MODE_NONE);
     CUtensorMap ma, mb;
     rc = encode_2d(&ma, A, K, M, lda, bk, kBM);
     if (rc != SPARQ_OK) return rc;
@@ -385,7 +399,7 @@ extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, in
         if (rc != 0) return rc < 0 ? rc : SPARQ_OK;
     }
     const int bk = (c % 128 == 0) ? 128 : 64;
-    const int bn = pick_bn(M, cout, sms);
+    const int bn = pick_bn(M, cout, sms, x.mode != SPARQ_MODE_NONE);
     CUtensorMap ma, mb;
     rc = encode_im2col(&ma, x_in, n, h, w, c, r, s, stride_h, stride_w, pad_h, pad_w, bk);
     if (rc != SPARQ_OK) return rc;
