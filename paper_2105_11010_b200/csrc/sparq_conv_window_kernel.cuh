@@ -202,10 +202,10 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         // ================= MMA issuer =================
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_i8(BN);
-            const uint64_t desc0 = make_smem_desc<CB>(smem_base);
-            const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
-            const uint32_t win_lo0 = (uint32_t)desc0;
-            const uint32_t b_lo0 = win_lo0 + (((uint32_t)g.win_bufs * win_bytes) >> 4);
+            // descriptors of window buffer 0 and of weight slot 0; offsets are added in units of
+            // 16 bytes to the start-address field (the low word never carries into the next field)
+            const uint64_t win_desc0 = make_smem_desc<CB>(smem_base);
+            const uint64_t b_desc0 = make_smem_desc<CB>(b_base);
             uint32_t wt = 0;
             int b = 0;  uint32_t wph = 0;      // window buffer and its phase parity
             int s = 0;  uint32_t bph = 0;      // streamed weight stage and its phase parity
@@ -224,24 +224,24 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 else SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b]), wph, abort_flag, g.status));
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                const uint32_t a_lo0 = win_lo0 + (uint32_t)b * (win_bytes >> 4);
+                const uint64_t a_desc0 = win_desc0 + (uint64_t)((uint32_t)b * (win_bytes >> 4));
                 const long long is0 = SPARQ_PROF_NOW();
                 // One (tap, channel block) of the tile: wait for its weights when they are
                 // streamed, then CB / 32 MMAs.
                 auto issue_block = [&](int kb, const uint2 e) {
-                    uint32_t b_lo;
+                    uint64_t bdesc;
                     if (B_RESIDENT) {
-                        b_lo = b_lo0 + e.y;
+                        bdesc = b_desc0 + (uint64_t)e.y;
                     } else {
                         SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status));
                         tc_fence_after();
-                        b_lo = b_lo0 + (uint32_t)s * (uint32_t)(kBBlock >> 4);
+                        bdesc = b_desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kBBlock >> 4));
                     }
-                    const uint32_t a_lo = a_lo0 + e.x;
+                    const uint64_t adesc = a_desc0 + (uint64_t)e.x;
 #pragma unroll
                     for (int k = 0; k < CB / 32; ++k)
-                        tc_mma_i8_parts(d_tmem, desc_hi, a_lo + (uint32_t)(k * 2), b_lo + (uint32_t)(k * 2), idesc,
-                                        (kb > 0 || k > 0) ? 1u : 0u);
+                        tc_mma_i8(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
+                                  (kb > 0 || k > 0) ? 1u : 0u);
                     if (!B_RESIDENT) {
                         tc_commit(smem_u32(&bar_b_empty[s]));
                         if (++s == g.b_stages) { s = 0; bph ^= 1u; }

@@ -185,21 +185,6 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint6
         :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
-// Same, with both descriptors given as (shared high word, low word): the high words of two
-// descriptors with the same row length and swizzle are equal, and the issuing thread then
-// only does 32-bit arithmetic per instruction.
-__device__ __forceinline__ void tc_mma_i8_parts(uint32_t d_tmem, uint32_t desc_hi, uint32_t a_lo, uint32_t b_lo,
-                                                uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "mov.b64 da, {%1, %3};\n\t"
-        "mov.b64 db, {%2, %3};\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t}"
-        :: "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
-}
-
 // Shared-memory matrix descriptor of a K-major tile whose rows are ROW_BYTES long
 // (128 or 64) and swizzled with the matching TMA mode; 8-row groups are contiguous.
 template <int ROW_BYTES>
@@ -517,10 +502,9 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         // ================= MMA issuer =================
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_i8(BN);
-            const uint64_t desc0 = make_smem_desc<BK>(smem_base);
-            const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
-            const uint32_t a_lo0 = (uint32_t)desc0;
-            const uint32_t b_lo0 = a_lo0 + (uint32_t)(Cfg::kABytes >> 4);
+            // descriptors of stage 0; a stage adds its byte offset / 16 to the start-address field
+            const uint64_t adesc0 = make_smem_desc<BK>(smem_base);
+            const uint64_t bdesc0 = make_smem_desc<BK>(smem_base + Cfg::kABytes);
             uint32_t local_tile = 0;
             int s = 0;             // stage
             uint32_t ph = 0;       // its phase parity
@@ -536,11 +520,12 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     if (MODE == SPARQ_MODE_NONE) SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_full[s]), ph, abort_flag, g.status));
                     else SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_xf[s]), ph, abort_flag, g.status));
                     tc_fence_after();
-                    const uint32_t st_off = (uint32_t)s * (uint32_t)(Cfg::kStageBytes >> 4);
+                    const uint64_t st_off = (uint64_t)((uint32_t)s * (uint32_t)(Cfg::kStageBytes >> 4));
+                    const uint64_t adesc = adesc0 + st_off, bdesc = bdesc0 + st_off;
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)
-                        tc_mma_i8_parts(d_tmem, desc_hi, a_lo0 + st_off + (uint32_t)(k * 2), b_lo0 + st_off + (uint32_t)(k * 2),
-                                        idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                        tc_mma_i8(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
+                                  (kb > 0 || k > 0) ? 1u : 0u);
                     tc_commit(smem_u32(&bar_empty[s]));       // stage reusable once these MMAs retire
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
