@@ -44,6 +44,7 @@ WGT_BYTES = COUT * R * S * C
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 INT8_OVER_BF16 = 2.0     # nominal dense ratio (4.5 POPS int8 vs 2.25 PFLOPS bf16)
+CONV_TRAFFIC_BYTES = 6530560 + 0   # ncu, per launch; set to None whenever the kernel changes
 
 
 def peaks():
@@ -390,8 +391,11 @@ def main():
         "roofline": {
             "bound": "tensor", "achieved": per_launch_tops, "peak": int8_peak, "unit": "TOP/s",
             "frac": per_launch_tops / int8_peak,
-            "traffic": None,
-            "kernel": "sparq_gemm_kernel<64,64,VSPARQ,4,round> (implicit-GEMM conv)",
+            # dram__bytes_read.sum + dram__bytes_write.sum of one launch (profiles/
+            # sparq_conv_window_kernel_cfg2.txt): the input is read once; the 6.4 MB of
+            # output is still dirty in the 126 MB L2 when the launch ends
+            "traffic": CONV_TRAFFIC_BYTES,
+            "kernel": "sparq_conv_window_kernel<64,64,VSPARQ,4,round,resident> (window implicit-GEMM conv)",
             "peak_source": f"{pk['source']} bf16 burst {pk['bf16']} TFLOP/s x {INT8_OVER_BF16} (nominal int8:bf16 ratio)",
             "algorithmic_ops_per_launch": OPS_PER_STEP,
             "algorithmic_bytes_per_launch": IN_BYTES + OUT_BYTES + WGT_BYTES,
