@@ -225,6 +225,24 @@ def cpu_baseline(images: int):
     return ops / dt / 1e12, dt, oracle.num_threads()
 
 
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """The slowest rank's time: every rank times the same K steps on its own shard, and the
+    job is as slow as its slowest replica.  Works on any initialized process group (NCCL on
+    GPUs, gloo in the CPU tests)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tops(ms_per_step: float, world: int) -> float:
+    """Weak scaling: each of the `world` replicas does one full workload per step."""
+    return world * OPS_PER_STEP / (ms_per_step * 1e-3) / 1e12
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -339,12 +357,9 @@ def main():
         sync()
     clocks = sampler.stop()
     sparq.sparq_check()
-    if world > 1:
-        t = torch.tensor([ms_total], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, device)
     ms_step = ms_total / args.steps
-    value = world * OPS_PER_STEP / (ms_step * 1e-3) / 1e12
+    value = whole_job_tops(ms_step, world)
 
     # end to end: pinned host input -> device -> fused kernel -> uint8 result back on the host
     x_host = torch.from_numpy(synth.activations(SEED, (NB, H, W, C), ZERO_FRAC, stream=10)).pin_memory()
@@ -364,11 +379,8 @@ def main():
     f1.record()
     sync(); barrier()
     e2e_ms = f0.elapsed_time(f1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * OPS_PER_STEP / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(e2e_ms, world, device)
+    e2e_value = whole_job_tops(e2e_ms / e2e_steps, world)
 
     int8_peak = pk["bf16"] * INT8_OVER_BF16
     per_launch_tops = OPS_PER_STEP / (ms_step * 1e-3) / 1e12

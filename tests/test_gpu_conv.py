@@ -67,6 +67,26 @@ def test_small_convolutions_exact(cfg, variant):
     check_full(x, wt, stride, pad, variant, seed=sum(cfg))
 
 
+@pytest.mark.parametrize("cfg", [
+    # shapes chosen to walk the stride-1 window kernel's paths and its fall-backs
+    (2, 30, 30, 384, 128, 3, 3, 1, 1),    # three channel blocks: 27 (tap, block) pairs, streamed weights
+    (3, 17, 23, 128, 200, 3, 3, 1, 1),    # cout not a tile multiple, rows not a multiple of the tile height
+    (1, 40, 20, 64, 64, 3, 3, 1, 1),      # tall image, 64-channel resident weights
+    (2, 14, 14, 256, 256, 3, 3, 1, 1),    # two channel blocks, partial last tile per image
+    (1, 8, 140, 64, 64, 3, 3, 1, 1),      # padded width above 128: im2col kernel
+    (1, 20, 20, 64, 64, 7, 7, 1, 3),      # 49 taps do not fit resident: im2col kernel
+    (2, 9, 9, 128, 128, 3, 3, 1, 0),      # no padding: output smaller than input
+    (2, 16, 16, 128, 128, 2, 2, 1, 1),    # even filter size
+    (4, 7, 7, 512, 512, 3, 3, 1, 1),      # 7x7 maps (too small for the window tiling)
+])
+def test_stride1_filter_shapes_exact(cfg):
+    nb, h, w, c, cout, r, s, stride, pad = cfg
+    x = synth.activations(sum(cfg) + 1, (nb, h, w, c), 0.5)
+    wt = synth.weights(sum(cfg) + 1, (cout, r, s, c))
+    for variant in (V5, (sparq.MODE_VSPARQ, 3, 0x29, 0)):
+        check_full(x, wt, stride, pad, variant, seed=sum(cfg))
+
+
 def test_config2_resnet18_conv_full():
     # 32 x 56 x 56 x 64, 45% zeros, 3x3 stride 1 pad 1, 64 filters; scale, bias, ReLU, requant
     x = synth.activations(1, (32, 56, 56, 64), 0.45)
