@@ -93,6 +93,13 @@ typedef struct {
     int32_t *acc_out;     /* raw accumulators, or NULL */
     float *f32_out;       /* dequantized fp32, or NULL */
     uint8_t *u8_out;      /* requantized activations for the next layer, or NULL */
+    /* Producer-side SPARQ.  The transform depends on the activations only (Section 3, first
+     * paragraph), so the layer that PRODUCES them can apply it once, and the consumer then
+     * runs with mode NONE at plain A8W8 speed.  If next_transform is non-NULL and its mode is
+     * not NONE, u8_out holds T(requantized row) with pairs (2j, 2j+1) along the N axis (the
+     * channels of an NHWC output, i.e. the next layer's reduction axis); acc_out and f32_out
+     * are unaffected.  Needs N to be a multiple of 4 (else SPARQ_ERR_UNSUPPORTED). */
+    const sparq_params *next_transform;   /* HOST pointer, or NULL */
 } sparq_epilogue;
 
 /* Standalone transform (Sections 3.1-3.2): out[r][k] = T(in[r][:])[k] for `rows` rows of

@@ -36,7 +36,7 @@ class _CEpilogue(ctypes.Structure):
     _fields_ = [("scale", ctypes.c_void_p), ("bias", ctypes.c_void_p),
                 ("relu", ctypes.c_int32), ("inv_out_scale", ctypes.c_float),
                 ("acc_out", ctypes.c_void_p), ("f32_out", ctypes.c_void_p),
-                ("u8_out", ctypes.c_void_p)]
+                ("u8_out", ctypes.c_void_p), ("next_transform", ctypes.POINTER(_CParams))]
 
 
 @dataclass(frozen=True)
@@ -142,21 +142,30 @@ def sparq_quantize(inp: torch.Tensor, out: torch.Tensor, rows: int, row_len: int
                                          rows, row_len, ctypes.byref(p), _stream_ptr(stream)))
 
 
-def _epilogue(n_cols: int, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out) -> _CEpilogue:
+def _next(next_transform):
+    """(pointer for the struct, object that keeps the pointee alive)"""
+    if next_transform is None:
+        return None, None
+    c = next_transform._c()
+    return ctypes.pointer(c), c
+
+
+def _epilogue(n_cols: int, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform=None) -> _CEpilogue:
     for name, t in (("scale", scale), ("bias", bias)):
         if t is not None and t.numel() < n_cols:
             raise ValueError(f"{name} has fewer than N elements")
     return _CEpilogue(_dev(scale, torch.float32, "scale"), _dev(bias, torch.float32, "bias"),
                       int(bool(relu)), float(inv_out_scale),
                       _dev(acc_out, torch.int32, "acc_out"), _dev(f32_out, torch.float32, "f32_out"),
-                      _dev(u8_out, torch.uint8, "u8_out"))
+                      _dev(u8_out, torch.uint8, "u8_out"), _next(next_transform)[0])
 
 
 def sparq_gemm_s8(A: torch.Tensor, B: torch.Tensor, params: SparqParams, *,
                   scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
                   relu: bool = False, inv_out_scale: float = 1.0,
                   acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
-                  u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+                  u8_out: Optional[torch.Tensor] = None,
+        next_transform: Optional[SparqParams] = None, stream=None) -> None:
     """``acc = T(A) @ B^T`` with A (M, K) uint8 and B (N, K) int8, then the epilogue."""
     M, K = A.shape
     N, K2 = B.shape
@@ -166,7 +175,7 @@ def sparq_gemm_s8(A: torch.Tensor, B: torch.Tensor, params: SparqParams, *,
         if t is not None and t.numel() < M * N:
             raise ValueError(f"{name} has fewer than M*N elements")
     p = params._c()
-    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out)
+    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform)
     _raise(load_library().sparq_gemm_s8(_dev(A, torch.uint8, "A"), K, _dev(B, torch.int8, "B"), K,
                                         M, N, K, ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))
 
@@ -175,7 +184,8 @@ def sparq_conv2d_nhwc_s8(x: torch.Tensor, w: torch.Tensor, stride, pad, params: 
                          scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
                          relu: bool = False, inv_out_scale: float = 1.0,
                          acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
-                         u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+                         u8_out: Optional[torch.Tensor] = None,
+        next_transform: Optional[SparqParams] = None, stream=None) -> None:
     """Fused convolution of NHWC uint8 ``x`` with [cout][r][s][c] int8 ``w``."""
     nb, h, wd, c = x.shape
     cout, r, s, c2 = w.shape
@@ -188,7 +198,7 @@ def sparq_conv2d_nhwc_s8(x: torch.Tensor, w: torch.Tensor, stride, pad, params: 
         if t is not None and t.numel() < m * cout:
             raise ValueError(f"{name} has fewer than N*Ho*Wo*Cout elements")
     p = params._c()
-    e = _epilogue(cout, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out)
+    e = _epilogue(cout, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform)
     _raise(load_library().sparq_conv2d_nhwc_s8(_dev(x, torch.uint8, "x"), nb, h, wd, c,
                                                _dev(w, torch.int8, "w"), cout, r, s,
                                                stride[0], stride[1], pad[0], pad[1],
@@ -273,7 +283,8 @@ def sparq_gemm_s8_static(A: torch.Tensor, B: torch.Tensor, params: SparqParams, 
                          scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
                          relu: bool = False, inv_out_scale: float = 1.0,
                          acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
-                         u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+                         u8_out: Optional[torch.Tensor] = None,
+        next_transform: Optional[SparqParams] = None, stream=None) -> None:
     """``sparq_gemm_s8`` for hosts that must not allocate device memory once running
     (all free memory already belongs to a framework's pool, or an allocation's
     device-wide synchronization is not acceptable).  Same result, computed as transform
@@ -289,6 +300,6 @@ def sparq_gemm_s8_static(A: torch.Tensor, B: torch.Tensor, params: SparqParams, 
         if t is not None and t.numel() < M * N:
             raise ValueError(f"{name} has fewer than M*N elements")
     p = params._c()
-    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out)
+    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform)
     _raise(load_library().sparq_gemm_s8_static(_dev(A, torch.uint8, "A"), K, _dev(B, torch.int8, "B"), K,
                                                M, N, K, ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))

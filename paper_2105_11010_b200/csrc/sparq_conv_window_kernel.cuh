@@ -48,6 +48,9 @@ struct WindowArgs {
     float *f32_out;
     uint8_t *u8_out;
     unsigned int *status;
+    // producer-side transform of u8_out (mode NONE = off)
+    int next_mode, next_rnd;
+    XformDev next_xf;
 };
 
 // dynamic shared memory the kernel may ask for: 227 KB minus room for its static variables

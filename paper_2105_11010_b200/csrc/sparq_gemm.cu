@@ -87,6 +87,24 @@ static int device_info(int *sms)
     return SPARQ_OK;
 }
 
+// Validates e->next_transform and turns it into kernel arguments (mode NONE when absent).
+static int next_transform_args(const sparq_epilogue *e, int64_t N, int *mode, int *rnd, XformDev *xf)
+{
+    *mode = SPARQ_MODE_NONE;
+    *rnd = 0;
+    *xf = XformDev{0u, 0, 4};
+    if (!e->next_transform || e->next_transform->mode == SPARQ_MODE_NONE) return SPARQ_OK;
+    XformArgs nx;
+    int rc = validate_params(e->next_transform, &nx);
+    if (rc != SPARQ_OK) return rc;
+    if (!e->u8_out) return set_error(SPARQ_ERR_INVALID_ARG, "next_transform needs u8_out");
+    if (N % 4) return set_error(SPARQ_ERR_UNSUPPORTED, "next_transform needs N (%lld) to be a multiple of 4", (long long)N);
+    *mode = nx.mode;
+    *rnd = nx.rnd;
+    *xf = XformDev{nx.widen_c, nx.widen_rounds, nx.n};
+    return SPARQ_OK;
+}
+
 static int check_epilogue(const sparq_epilogue *e)
 {
     if (!e) return set_error(SPARQ_ERR_INVALID_ARG, "sparq_epilogue is NULL");
@@ -145,7 +163,7 @@ static cudaError_t launch(int bn, int bk, const CUtensorMap &ma, const CUtensorM
     return launch_gemm_shape<256, 128>(ma, mb, g, x.mode, variant_n(x), x.rnd, grid, st);
 }
 
-static void fill_common(GemmArgs *g, const XformArgs &x, const sparq_epilogue *e, unsigned int *status)
+static int fill_common(GemmArgs *g, const XformArgs &x, const sparq_epilogue *e, unsigned int *status)
 {
     g->xf = XformDev{x.widen_c, x.widen_rounds, x.n};
     g->scale = e->scale;
@@ -156,6 +174,7 @@ static void fill_common(GemmArgs *g, const XformArgs &x, const sparq_epilogue *e
     g->f32_out = e->f32_out;
     g->u8_out = e->u8_out;
     g->status = status;
+    return next_transform_args(e, g->N, &g->next_mode, &g->next_rnd, &g->next_xf);
 }
 
 static int gemm_impl(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb, int64_t M, int64_t N, int64_t K,
@@ -183,7 +202,8 @@ static int gemm_impl(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     memset(&g, 0, sizeof(g));
     g.M = M; g.N = N; g.K = K;
     g.k_blocks = (int)((K + bk - 1) / bk);
-    fill_common(&g, x, e, status);
+    rc = fill_common(&g, x, e, status);
+    if (rc != SPARQ_OK) return rc;
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
     const int grid = (int)(tiles < sms ? tiles : sms);
     cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
@@ -291,6 +311,8 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     g.scale = e->scale; g.bias = e->bias; g.relu = e->relu ? 1 : 0; g.inv_out_scale = e->inv_out_scale;
     g.acc_out = e->acc_out; g.f32_out = e->f32_out; g.u8_out = e->u8_out;
     g.status = status;
+    rc = next_transform_args(e, g.N, &g.next_mode, &g.next_rnd, &g.next_xf);
+    if (rc != SPARQ_OK) return rc;
     const int64_t tiles = m_tiles * n_tiles;
     const int grid = (int)(tiles < sms ? tiles : sms);
     cudaError_t ce;
@@ -322,7 +344,8 @@ int gemm_with_status(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     memset(&g, 0, sizeof(g));
     g.M = M; g.N = N; g.K = K;
     g.k_blocks = (int)((K + bk - 1) / bk);
-    fill_common(&g, x, e, status);
+    rc = fill_common(&g, x, e, status);
+    if (rc != SPARQ_OK) return rc;
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
     const int grid = (int)(tiles < sms ? tiles : sms);
     cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
@@ -414,7 +437,8 @@ extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, in
     g.S = s;
     g.Ho = ho; g.Wo = wo;
     g.stride_h = stride_h; g.stride_w = stride_w; g.pad_h = pad_h; g.pad_w = pad_w;
-    fill_common(&g, x, e, status);
+    rc = fill_common(&g, x, e, status);
+    if (rc != SPARQ_OK) return rc;
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((cout + bn - 1) / bn);
     const int grid = (int)(tiles < sms ? tiles : sms);
     cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);

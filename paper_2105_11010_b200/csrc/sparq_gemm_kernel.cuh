@@ -75,6 +75,9 @@ struct GemmArgs {
     float *f32_out;
     uint8_t *u8_out;
     unsigned int *status;
+    // producer-side transform of u8_out (mode NONE = off)
+    int next_mode, next_rnd;
+    XformDev next_xf;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------
@@ -278,6 +281,9 @@ struct EpiView {
     bool small_acc;   // |acc| < 2^22 guaranteed
     bool vec_ok;      // rows allow 16/32-byte vector stores
     bool u8_wide;     // 256-bit stores allowed on u8_out
+    int next_mode;    // SPARQ mode applied to the requantized bytes (producer-side transform)
+    int next_rnd;
+    XformDev next_xf;
 };
 
 template <class Args>
@@ -298,6 +304,9 @@ __device__ __forceinline__ EpiView make_epi_view(const Args &g)
     e.small_acc = g.K * (255 * 128) < (1 << 22);
     e.vec_ok = (g.N % 32) == 0;
     e.u8_wide = (reinterpret_cast<uintptr_t>(g.u8_out) & 31u) == 0;
+    e.next_mode = g.next_mode;
+    e.next_rnd = g.next_rnd;
+    e.next_xf = g.next_xf;
     return e;
 }
 
@@ -354,6 +363,19 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[32], i
                          requant_bits(__uint_as_float(v[4 * q + 1]), e.inv_out_scale),
                          requant_bits(__uint_as_float(v[4 * q + 2]), e.inv_out_scale),
                          requant_bits(__uint_as_float(v[4 * q + 3]), e.inv_out_scale));
+        if (e.next_mode != SPARQ_MODE_NONE) {
+            // the next layer's transform on the bytes just produced: four adjacent output
+            // channels per word, pairs (2j, 2j+1) inside it (general run-time-width form)
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                if (e.next_mode == SPARQ_MODE_VSPARQ)
+                    w[q] = e.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 0, true, true>(w[q], e.next_xf)
+                                      : xform_word<SPARQ_MODE_VSPARQ, 0, false, true>(w[q], e.next_xf);
+                else
+                    w[q] = e.next_rnd ? xform_word<SPARQ_MODE_BSPARQ, 0, true, true>(w[q], e.next_xf)
+                                      : xform_word<SPARQ_MODE_BSPARQ, 0, false, true>(w[q], e.next_xf);
+            }
+        }
         if (full && e.u8_wide) {
             st_global_v8(e.u8_out + off, w);
         } else if (full) {
