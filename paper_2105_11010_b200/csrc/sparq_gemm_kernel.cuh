@@ -365,15 +365,21 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[32], i
                          requant_bits(__uint_as_float(v[4 * q + 3]), e.inv_out_scale));
         if (e.next_mode != SPARQ_MODE_NONE) {
             // the next layer's transform on the bytes just produced: four adjacent output
-            // channels per word, pairs (2j, 2j+1) inside it (general run-time-width form)
+            // channels per word, pairs (2j, 2j+1) inside it
+            const bool fast4 = e.next_xf.n == 4 && e.next_xf.rounds == 0;   // n = 4, all five placements
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
-                if (e.next_mode == SPARQ_MODE_VSPARQ)
-                    w[q] = e.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 0, true, true>(w[q], e.next_xf)
-                                      : xform_word<SPARQ_MODE_VSPARQ, 0, false, true>(w[q], e.next_xf);
-                else
-                    w[q] = e.next_rnd ? xform_word<SPARQ_MODE_BSPARQ, 0, true, true>(w[q], e.next_xf)
-                                      : xform_word<SPARQ_MODE_BSPARQ, 0, false, true>(w[q], e.next_xf);
+                if (e.next_mode == SPARQ_MODE_VSPARQ) {
+                    if (fast4) w[q] = e.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 4, true, false>(w[q], e.next_xf)
+                                                 : xform_word<SPARQ_MODE_VSPARQ, 4, false, false>(w[q], e.next_xf);
+                    else w[q] = e.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 0, true, true>(w[q], e.next_xf)
+                                           : xform_word<SPARQ_MODE_VSPARQ, 0, false, true>(w[q], e.next_xf);
+                } else {
+                    if (fast4) w[q] = e.next_rnd ? xform_word<SPARQ_MODE_BSPARQ, 4, true, false>(w[q], e.next_xf)
+                                                 : xform_word<SPARQ_MODE_BSPARQ, 4, false, false>(w[q], e.next_xf);
+                    else w[q] = e.next_rnd ? xform_word<SPARQ_MODE_BSPARQ, 0, true, true>(w[q], e.next_xf)
+                                           : xform_word<SPARQ_MODE_BSPARQ, 0, false, true>(w[q], e.next_xf);
+                }
             }
         }
         if (full && e.u8_wide) {
