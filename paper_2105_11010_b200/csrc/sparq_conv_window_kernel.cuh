@@ -144,15 +144,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            if (B_RESIDENT) {
-                // all weight blocks, once per CTA, on stage barrier 0
-                const uint32_t full = smem_u32(&bar_b_full[0]);
-                mbar_expect_tx(full, (uint32_t)kb_count * kBBlock);
-                for (int kb = 0; kb < kb_count; ++kb) {
-                    const int cb = kb / taps, tap = kb % taps;
-                    tma_load_2d(b_slot(kb), &map_w, full, tap * g.C + cb * CB, 0);
-                }
-            }
             uint32_t wt = 0;      // window counter
             uint32_t it = 0;      // streamed weight-block counter
             long long pw = 0;
@@ -170,6 +161,17 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 for (int cb = 0; cb < g.c_blocks; ++cb)
                     tma_load_4d(win_buf(b) + (uint32_t)cb * g.plane_bytes, &map_x, wfull,
                                 cb * CB, -g.pad_w, oh0 - g.pad_h, img);
+                if (B_RESIDENT && wt == 0) {
+                    // all weight blocks, once per CTA, on stage barrier 0 -- after the first
+                    // window so that the activations (which come from HBM and still have to
+                    // be transformed) are requested first
+                    const uint32_t full = smem_u32(&bar_b_full[0]);
+                    mbar_expect_tx(full, (uint32_t)kb_count * kBBlock);
+                    for (int kb = 0; kb < kb_count; ++kb) {
+                        const int cb = kb / taps, tap = kb % taps;
+                        tma_load_2d(b_slot(kb), &map_w, full, tap * g.C + cb * CB, 0);
+                    }
+                }
                 if (!B_RESIDENT) {
                     for (int kb = 0; kb < kb_count; ++kb, ++it) {
                         const int s = it % g.b_stages;
@@ -192,7 +194,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 for (uint32_t j = wfirst; j < wt; ++j)
                     mbar_wait(smem_u32(&bar_win_full[j % g.win_bufs]), (j / g.win_bufs) & 1, abort_flag, g.status, true);
                 if (B_RESIDENT) {
-                    mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, true);
+                    // the weight copies were issued together with the first window
+                    if (wt > 0) mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, true);
                 } else {
                     const uint32_t first = it > (uint32_t)g.b_stages ? it - g.b_stages : 0;
                     for (uint32_t j = first; j < it; ++j)
