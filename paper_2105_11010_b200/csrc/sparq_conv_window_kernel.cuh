@@ -146,6 +146,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         if (lane == 0) {
             uint32_t wt = 0;      // window counter
             uint32_t it = 0;      // streamed weight-block counter
+            bool b_issued = false;  // resident weights requested
             long long pw = 0;
             const long long pt0 = SPARQ_PROF_NOW();
             for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
@@ -171,6 +172,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                         const int cb = kb / taps, tap = kb % taps;
                         tma_load_2d(b_slot(kb), &map_w, full, tap * g.C + cb * CB, 0);
                     }
+                    b_issued = true;
                 }
                 if (!B_RESIDENT) {
                     for (int kb = 0; kb < kb_count; ++kb, ++it) {
@@ -195,7 +197,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                     mbar_wait(smem_u32(&bar_win_full[j % g.win_bufs]), (j / g.win_bufs) & 1, abort_flag, g.status, true);
                 if (B_RESIDENT) {
                     // the weight copies were issued together with the first window
-                    if (wt > 0) mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, true);
+                    if (b_issued) mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, true);
                 } else {
                     const uint32_t first = it > (uint32_t)g.b_stages ? it - g.b_stages : 0;
                     for (uint32_t j = first; j < it; ++j)
