@@ -186,7 +186,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                         tma_load_2d(b_slot(s), &map_w, full, tap * g.C + cb * CB, (int)(nt * BN));
                     }
                 }
-                if (*abort_flag) break;
+                // an abort noticed here is acted on at the top of the next iteration, after this
+                // tile's window has been counted in wt (the drain below waits for it)
             }
             SPARQ_PROF_STORE(0, pw);
             SPARQ_PROF_STORE(1, SPARQ_PROF_NOW() - pt0);
