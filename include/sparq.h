@@ -39,7 +39,7 @@ extern "C" {
 typedef enum {
     SPARQ_OK = 0,
     SPARQ_ERR_INVALID_ARG = -1, /* null pointer, negative size, bad mode / width / placement set */
-    SPARQ_ERR_UNSUPPORTED = -2, /* a shape or alignment this build has no kernel for */
+    SPARQ_ERR_UNSUPPORTED = -2, /* a shape or alignment the library has no kernel for */
     SPARQ_ERR_CUDA = -3,        /* a CUDA runtime / driver call failed (text in sparq_last_error) */
     SPARQ_ERR_TIMEOUT = -4      /* a bounded device-side wait expired (reported by sparq_check) */
 } sparq_status;
