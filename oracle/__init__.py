@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_conv2d_nhwc.restype = None
         L.oracle_epilogue.argtypes = [p, i64, i64, p, p, i, f32, p, p]
         L.oracle_epilogue.restype = None
+        L.oracle_epilogue_residual.argtypes = [p, i64, i64, p, p, p, f32, i, f32, p, p]
+        L.oracle_epilogue_residual.restype = None
         L.oracle_num_threads.restype = i
         L.oracle_set_num_threads.argtypes = [i]
         _lib = L
@@ -159,9 +161,11 @@ def conv2d_nhwc(x: np.ndarray, w: np.ndarray, stride: Tuple[int, int], pad: Tupl
 
 
 def epilogue(acc: np.ndarray, scale: np.ndarray, bias: Optional[np.ndarray], relu: bool,
-             inv_out_scale: float) -> Tuple[np.ndarray, np.ndarray]:
+             inv_out_scale: float, residual: Optional[np.ndarray] = None,
+             residual_scale: float = 0.0) -> Tuple[np.ndarray, np.ndarray]:
     """(fp32 output, requantized uint8 output) of the int32 accumulators; the
-    channel axis is the last one."""
+    channel axis is the last one.  `residual` (uint8, same shape) times
+    `residual_scale` is added before the ReLU."""
     acc = _c(acc, np.int32)
     N = acc.shape[-1]
     M = acc.size // N if N else 0
@@ -169,9 +173,13 @@ def epilogue(acc: np.ndarray, scale: np.ndarray, bias: Optional[np.ndarray], rel
     b = None if bias is None else _c(bias, np.float32)
     f = np.empty(acc.shape, dtype=np.float32)
     q = np.empty(acc.shape, dtype=np.uint8)
+    r = None if residual is None else _c(residual, np.uint8)
+    if r is not None and r.shape != acc.shape:
+        raise ValueError("residual must have the accumulators' shape")
     if acc.size:
-        lib().oracle_epilogue(_ptr(acc), M, N, _ptr(scale), _ptr(b), int(bool(relu)),
-                              ctypes.c_float(inv_out_scale), _ptr(f), _ptr(q))
+        lib().oracle_epilogue_residual(_ptr(acc), M, N, _ptr(scale), _ptr(b), _ptr(r),
+                                       ctypes.c_float(residual_scale), int(bool(relu)),
+                                       ctypes.c_float(inv_out_scale), _ptr(f), _ptr(q))
     return f, q
 
 

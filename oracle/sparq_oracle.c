@@ -244,19 +244,28 @@ void oracle_conv2d_nhwc(const uint8_t *x, int nb, int h, int w, int c,
  * fp32 sequence, one IEEE operation per line, no contraction:
  *     t = (float)acc                       int32 -> fp32, round to nearest even
  *     y = fma(t, scale[j], bias[j])        single rounding
+ *     y = fma((float)res, res_scale, y)    only with a residual input: the block's u8
+ *                                          identity tensor on its own scale, added before
+ *                                          the ReLU as in a ResNet bottleneck
  *     y = relu ? max(y, 0) : y             (y > 0 ? y : 0)
  *     z = y * inv_out_scale
  *     u = rint(z)                          nearest even
  *     q = clamp(u, 0, 255) as uint8        NaN -> 0
- * Any of f32_out / u8_out may be NULL. */
-void oracle_epilogue(const int32_t *acc, int64_t M, int64_t N,
-                     const float *scale, const float *bias, int relu, float inv_out_scale,
-                     float *f32_out, uint8_t *u8_out)
+ * Any of f32_out / u8_out may be NULL; residual may be NULL (no residual step). */
+void oracle_epilogue_residual(const int32_t *acc, int64_t M, int64_t N,
+                              const float *scale, const float *bias,
+                              const uint8_t *residual, float residual_scale,
+                              int relu, float inv_out_scale,
+                              float *f32_out, uint8_t *u8_out)
 {
     for (int64_t m = 0; m < M; ++m) {
         for (int64_t j = 0; j < N; ++j) {
             volatile float t = (float)acc[m * N + j];
             volatile float y = fmaf(t, scale[j], bias ? bias[j] : 0.0f);
+            if (residual) {
+                volatile float r = (float)residual[m * N + j];
+                y = fmaf(r, residual_scale, y);
+            }
             if (relu) y = (y > 0.0f) ? y : 0.0f;
             if (f32_out) f32_out[m * N + j] = y;
             if (u8_out) {
@@ -270,6 +279,13 @@ void oracle_epilogue(const int32_t *acc, int64_t M, int64_t N,
             }
         }
     }
+}
+
+void oracle_epilogue(const int32_t *acc, int64_t M, int64_t N,
+                     const float *scale, const float *bias, int relu, float inv_out_scale,
+                     float *f32_out, uint8_t *u8_out)
+{
+    oracle_epilogue_residual(acc, M, N, scale, bias, NULL, 0.0f, relu, inv_out_scale, f32_out, u8_out);
 }
 
 int oracle_num_threads(void)

@@ -150,3 +150,43 @@ def test_epilogue_rounding_and_saturation_cases():
     f, q = oracle.epilogue(acc, scale, None, False, 1.0)
     assert list(f[0]) == [0.5, 1.5, 2.5, 500.0, -3.5, 1.0]
     assert list(q[0]) == [0, 2, 2, 255, 0, 1]      # ties to even, clamp to [0, 255]
+
+
+def test_epilogue_residual_against_float64():
+    # y = acc*scale + bias + residual*residual_scale, then ReLU: the float64 value bounds the
+    # fp32 result (three roundings), the residual is added BEFORE the ReLU, and a NULL
+    # residual or a zero residual tensor leaves the plain epilogue.
+    rng = np.random.default_rng(5)
+    acc = rng.integers(-300_000, 300_000, size=(32, 40), dtype=np.int64).astype(np.int32)
+    scale = synth.scales(2, 40)
+    b = synth.bias(2, 40)
+    res = rng.integers(0, 256, size=(32, 40), dtype=np.uint8)
+    rs = np.float32(0.37)
+    inv = np.float32(1.0 / 9.0)
+    for relu in (False, True):
+        f, q = oracle.epilogue(acc, scale, b, relu, inv, residual=res, residual_scale=rs)
+        part = acc.astype(np.float64) * scale + b
+        y64 = part + res.astype(np.float64) * np.float64(rs)
+        if relu:
+            y64 = np.maximum(y64, 0)
+        bound = 1.3e-7 * (np.abs(acc.astype(np.float64) * scale) + np.abs(part)
+                          + np.abs(res * np.float64(rs)) + np.abs(y64)) + 1e-30
+        assert (np.abs(f - y64) <= bound).all()
+        assert np.array_equal(q, np.clip(np.rint(f * inv), 0, 255).astype(np.uint8))
+        f0, q0 = oracle.epilogue(acc, scale, b, relu, inv)
+        fz, qz = oracle.epilogue(acc, scale, b, relu, inv, residual=np.zeros_like(res), residual_scale=rs)
+        assert np.array_equal(f0, fz) and np.array_equal(q0, qz)
+        assert not np.array_equal(f0, f)
+
+
+def test_epilogue_residual_exact_cases():
+    # values exact in fp32: (acc*0.5 + 1) + res*0.25, ReLU after the sum
+    acc = np.array([[-10, -10, 4, 0]], dtype=np.int32)
+    scale = np.full(4, 0.5, np.float32)
+    bias = np.ones(4, np.float32)
+    res = np.array([[8, 32, 2, 255]], dtype=np.uint8)
+    f, q = oracle.epilogue(acc, scale, bias, True, 1.0, residual=res, residual_scale=0.25)
+    assert list(f[0]) == [0.0, 4.0, 3.5, 64.75]       # -4+2 -> ReLU 0 ; -4+8 ; 3+0.5 ; 1+63.75
+    assert list(q[0]) == [0, 4, 4, 65]
+    f, _ = oracle.epilogue(acc, scale, bias, False, 1.0, residual=res, residual_scale=0.25)
+    assert f[0, 0] == -2.0
