@@ -80,7 +80,9 @@ typedef struct {
 /* What happens to the int32 accumulators (not in the paper beyond its quantization
  * scheme, Section 5: per-layer activation scale times per-kernel weight scale).  For
  * output column j, in fp32 and in this order, one IEEE operation each:
- *     t = (float)acc;  y = fma(t, scale[j], bias ? bias[j] : 0);  if (relu) y = y > 0 ? y : 0;
+ *     t = (float)acc;  y = fma(t, scale[j], bias ? bias[j] : 0);
+ *     if (residual) y = fma((float)residual[m][j], residual_scale, y);
+ *     if (relu) y = y > 0 ? y : 0;
  *     f32_out = y;     u8_out = clamp(rint(y * inv_out_scale), 0, 255)   (NaN -> 0)
  * Each output pointer may be NULL (that output is not produced); at least one must be
  * non-NULL.  Outputs are M x N row-major with leading dimension N (= NHWC for the
@@ -100,6 +102,15 @@ typedef struct {
      * channels of an NHWC output, i.e. the next layer's reduction axis); acc_out and f32_out
      * are unaffected.  Needs N to be a multiple of 4 (else SPARQ_ERR_UNSUPPORTED). */
     const sparq_params *next_transform;   /* HOST pointer, or NULL */
+    /* Residual input: the u8 identity tensor of a residual block (M x N row-major like the
+     * outputs, on its own scale), added before the ReLU so that the last convolution of a
+     * bottleneck writes the block's output in one pass.  Not in the paper, whose transform
+     * acts on whatever activations a layer receives.  NULL = no residual.  Must be 16-byte
+     * aligned (else SPARQ_ERR_UNSUPPORTED), needs scale (a dequantized output), and may be
+     * the same buffer as u8_out only if every row is read before it is written, which this
+     * library does not promise: pass distinct buffers. */
+    const uint8_t *residual;              /* [M x N] device, or NULL */
+    float residual_scale;
 } sparq_epilogue;
 
 /* Standalone transform (Sections 3.1-3.2): out[r][k] = T(in[r][:])[k] for `rows` rows of
@@ -153,7 +164,7 @@ SPARQ_API int sparq_quantize_host(const uint8_t *in_host, uint8_t *out_host, siz
                         const sparq_params *p, void *stream);
 
 /* A_host: HOST, M x K with leading dimension lda.  B: DEVICE.  In `e`, scale and bias are
- * DEVICE pointers and acc_out / f32_out / u8_out are HOST pointers (M x N each). */
+ * DEVICE pointers and acc_out / f32_out / u8_out / residual are HOST pointers (M x N each). */
 SPARQ_API int sparq_gemm_s8_host(const uint8_t *A_host, int64_t lda, const int8_t *B, int64_t ldb,
                        int64_t M, int64_t N, int64_t K,
                        const sparq_params *p, const sparq_epilogue *e, void *stream);

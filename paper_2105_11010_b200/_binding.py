@@ -36,7 +36,8 @@ class _CEpilogue(ctypes.Structure):
     _fields_ = [("scale", ctypes.c_void_p), ("bias", ctypes.c_void_p),
                 ("relu", ctypes.c_int32), ("inv_out_scale", ctypes.c_float),
                 ("acc_out", ctypes.c_void_p), ("f32_out", ctypes.c_void_p),
-                ("u8_out", ctypes.c_void_p), ("next_transform", ctypes.POINTER(_CParams))]
+                ("u8_out", ctypes.c_void_p), ("next_transform", ctypes.POINTER(_CParams)),
+                ("residual", ctypes.c_void_p), ("residual_scale", ctypes.c_float)]
 
 
 @dataclass(frozen=True)
@@ -150,14 +151,16 @@ def _next(next_transform):
     return ctypes.pointer(c), c
 
 
-def _epilogue(n_cols: int, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform=None) -> _CEpilogue:
+def _epilogue(n_cols: int, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform=None,
+              residual=None, residual_scale=0.0) -> _CEpilogue:
     for name, t in (("scale", scale), ("bias", bias)):
         if t is not None and t.numel() < n_cols:
             raise ValueError(f"{name} has fewer than N elements")
     return _CEpilogue(_dev(scale, torch.float32, "scale"), _dev(bias, torch.float32, "bias"),
                       int(bool(relu)), float(inv_out_scale),
                       _dev(acc_out, torch.int32, "acc_out"), _dev(f32_out, torch.float32, "f32_out"),
-                      _dev(u8_out, torch.uint8, "u8_out"), _next(next_transform)[0])
+                      _dev(u8_out, torch.uint8, "u8_out"), _next(next_transform)[0],
+                      _dev(residual, torch.uint8, "residual"), float(residual_scale))
 
 
 def sparq_gemm_s8(A: torch.Tensor, B: torch.Tensor, params: SparqParams, *,
@@ -165,17 +168,19 @@ def sparq_gemm_s8(A: torch.Tensor, B: torch.Tensor, params: SparqParams, *,
                   relu: bool = False, inv_out_scale: float = 1.0,
                   acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
                   u8_out: Optional[torch.Tensor] = None,
-        next_transform: Optional[SparqParams] = None, stream=None) -> None:
+                  next_transform: Optional[SparqParams] = None,
+                  residual: Optional[torch.Tensor] = None, residual_scale: float = 0.0, stream=None) -> None:
     """``acc = T(A) @ B^T`` with A (M, K) uint8 and B (N, K) int8, then the epilogue."""
     M, K = A.shape
     N, K2 = B.shape
     if K != K2:
         raise ValueError("A and B disagree on K")
-    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out)):
+    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out), ("residual", residual)):
         if t is not None and t.numel() < M * N:
             raise ValueError(f"{name} has fewer than M*N elements")
     p = params._c()
-    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform)
+    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform,
+                  residual, residual_scale)
     _raise(load_library().sparq_gemm_s8(_dev(A, torch.uint8, "A"), K, _dev(B, torch.int8, "B"), K,
                                         M, N, K, ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))
 
@@ -185,7 +190,8 @@ def sparq_conv2d_nhwc_s8(x: torch.Tensor, w: torch.Tensor, stride, pad, params: 
                          relu: bool = False, inv_out_scale: float = 1.0,
                          acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
                          u8_out: Optional[torch.Tensor] = None,
-        next_transform: Optional[SparqParams] = None, stream=None) -> None:
+                  next_transform: Optional[SparqParams] = None,
+                  residual: Optional[torch.Tensor] = None, residual_scale: float = 0.0, stream=None) -> None:
     """Fused convolution of NHWC uint8 ``x`` with [cout][r][s][c] int8 ``w``."""
     nb, h, wd, c = x.shape
     cout, r, s, c2 = w.shape
@@ -194,11 +200,12 @@ def sparq_conv2d_nhwc_s8(x: torch.Tensor, w: torch.Tensor, stride, pad, params: 
     ho = (h + 2 * pad[0] - r) // stride[0] + 1
     wo = (wd + 2 * pad[1] - s) // stride[1] + 1
     m = nb * ho * wo
-    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out)):
+    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out), ("residual", residual)):
         if t is not None and t.numel() < m * cout:
             raise ValueError(f"{name} has fewer than N*Ho*Wo*Cout elements")
     p = params._c()
-    e = _epilogue(cout, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform)
+    e = _epilogue(cout, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform,
+                  residual, residual_scale)
     _raise(load_library().sparq_conv2d_nhwc_s8(_dev(x, torch.uint8, "x"), nb, h, wd, c,
                                                _dev(w, torch.int8, "w"), cout, r, s,
                                                stride[0], stride[1], pad[0], pad[1],
@@ -231,20 +238,22 @@ def sparq_gemm_s8_host(A: torch.Tensor, B: torch.Tensor, params: SparqParams, *,
                        scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
                        relu: bool = False, inv_out_scale: float = 1.0,
                        acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
-                       u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+                       u8_out: Optional[torch.Tensor] = None,
+                  residual: Optional[torch.Tensor] = None, residual_scale: float = 0.0, stream=None) -> None:
     """Host-buffer form of :func:`sparq_gemm_s8`: ``A`` and the outputs are CPU tensors."""
     M, K = A.shape
     N, K2 = B.shape
     if K != K2:
         raise ValueError("A and B disagree on K")
-    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out)):
+    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out), ("residual", residual)):
         if t is not None and t.numel() < M * N:
             raise ValueError(f"{name} has fewer than M*N elements")
     p = params._c()
     e = _CEpilogue(_dev(scale, torch.float32, "scale"), _dev(bias, torch.float32, "bias"),
                    int(bool(relu)), float(inv_out_scale),
                    _host(acc_out, torch.int32, "acc_out"), _host(f32_out, torch.float32, "f32_out"),
-                   _host(u8_out, torch.uint8, "u8_out"))
+                   _host(u8_out, torch.uint8, "u8_out"), None,
+                   _host(residual, torch.uint8, "residual"), float(residual_scale))
     _raise(load_library().sparq_gemm_s8_host(_host(A, torch.uint8, "A"), K, _dev(B, torch.int8, "B"), K,
                                              M, N, K, ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))
 
@@ -253,7 +262,8 @@ def sparq_conv2d_nhwc_s8_host(x: torch.Tensor, w: torch.Tensor, stride, pad, par
                               scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
                               relu: bool = False, inv_out_scale: float = 1.0,
                               acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
-                              u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+                              u8_out: Optional[torch.Tensor] = None,
+                  residual: Optional[torch.Tensor] = None, residual_scale: float = 0.0, stream=None) -> None:
     """Host-buffer form of :func:`sparq_conv2d_nhwc_s8`: ``x`` and the outputs are CPU tensors."""
     nb, h, wd, c = x.shape
     cout, r, s, c2 = w.shape
@@ -262,14 +272,15 @@ def sparq_conv2d_nhwc_s8_host(x: torch.Tensor, w: torch.Tensor, stride, pad, par
     ho = (h + 2 * pad[0] - r) // stride[0] + 1
     wo = (wd + 2 * pad[1] - s) // stride[1] + 1
     m = nb * ho * wo
-    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out)):
+    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out), ("residual", residual)):
         if t is not None and t.numel() < m * cout:
             raise ValueError(f"{name} has fewer than N*Ho*Wo*Cout elements")
     p = params._c()
     e = _CEpilogue(_dev(scale, torch.float32, "scale"), _dev(bias, torch.float32, "bias"),
                    int(bool(relu)), float(inv_out_scale),
                    _host(acc_out, torch.int32, "acc_out"), _host(f32_out, torch.float32, "f32_out"),
-                   _host(u8_out, torch.uint8, "u8_out"))
+                   _host(u8_out, torch.uint8, "u8_out"), None,
+                   _host(residual, torch.uint8, "residual"), float(residual_scale))
     _raise(load_library().sparq_conv2d_nhwc_s8_host(_host(x, torch.uint8, "x"), nb, h, wd, c,
                                                     _dev(w, torch.int8, "w"), cout, r, s,
                                                     stride[0], stride[1], pad[0], pad[1],
@@ -284,7 +295,8 @@ def sparq_gemm_s8_static(A: torch.Tensor, B: torch.Tensor, params: SparqParams, 
                          relu: bool = False, inv_out_scale: float = 1.0,
                          acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
                          u8_out: Optional[torch.Tensor] = None,
-        next_transform: Optional[SparqParams] = None, stream=None) -> None:
+                  next_transform: Optional[SparqParams] = None,
+                  residual: Optional[torch.Tensor] = None, residual_scale: float = 0.0, stream=None) -> None:
     """``sparq_gemm_s8`` for hosts that must not allocate device memory once running
     (all free memory already belongs to a framework's pool, or an allocation's
     device-wide synchronization is not acceptable).  Same result, computed as transform
@@ -296,10 +308,11 @@ def sparq_gemm_s8_static(A: torch.Tensor, B: torch.Tensor, params: SparqParams, 
     N, K2 = B.shape
     if K != K2:
         raise ValueError("A and B disagree on K")
-    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out)):
+    for name, t in (("acc_out", acc_out), ("f32_out", f32_out), ("u8_out", u8_out), ("residual", residual)):
         if t is not None and t.numel() < M * N:
             raise ValueError(f"{name} has fewer than M*N elements")
     p = params._c()
-    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform)
+    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out, next_transform,
+                  residual, residual_scale)
     _raise(load_library().sparq_gemm_s8_static(_dev(A, torch.uint8, "A"), K, _dev(B, torch.int8, "B"), K,
                                                M, N, K, ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))

@@ -51,6 +51,8 @@ struct WindowArgs {
     // producer-side transform of u8_out (mode NONE = off)
     int next_mode, next_rnd;
     XformDev next_xf;
+    const uint8_t *residual;
+    float residual_scale;
 };
 
 // dynamic shared memory the kernel may ask for: 227 KB minus room for its static variables

@@ -115,6 +115,12 @@ static int check_epilogue(const sparq_epilogue *e)
     if ((e->acc_out && ((uintptr_t)e->acc_out & 15u)) || (e->f32_out && ((uintptr_t)e->f32_out & 15u)) ||
         (e->u8_out && ((uintptr_t)e->u8_out & 15u)))
         return set_error(SPARQ_ERR_UNSUPPORTED, "output pointers must be 16-byte aligned");
+    if (e->residual) {
+        if (!e->f32_out && !e->u8_out)
+            return set_error(SPARQ_ERR_INVALID_ARG, "residual needs a dequantized output (f32_out or u8_out)");
+        if ((uintptr_t)e->residual & 15u)
+            return set_error(SPARQ_ERR_UNSUPPORTED, "residual must be 16-byte aligned");
+    }
     return SPARQ_OK;
 }
 
@@ -174,6 +180,8 @@ static int fill_common(GemmArgs *g, const XformArgs &x, const sparq_epilogue *e,
     g->f32_out = e->f32_out;
     g->u8_out = e->u8_out;
     g->status = status;
+    g->residual = e->residual;
+    g->residual_scale = e->residual_scale;
     return next_transform_args(e, g->N, &g->next_mode, &g->next_rnd, &g->next_xf);
 }
 
@@ -311,6 +319,8 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     g.scale = e->scale; g.bias = e->bias; g.relu = e->relu ? 1 : 0; g.inv_out_scale = e->inv_out_scale;
     g.acc_out = e->acc_out; g.f32_out = e->f32_out; g.u8_out = e->u8_out;
     g.status = status;
+    g.residual = e->residual;
+    g.residual_scale = e->residual_scale;
     rc = next_transform_args(e, g.N, &g.next_mode, &g.next_rnd, &g.next_xf);
     if (rc != SPARQ_OK) return rc;
     const int64_t tiles = m_tiles * n_tiles;

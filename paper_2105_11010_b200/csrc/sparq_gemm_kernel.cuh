@@ -78,6 +78,9 @@ struct GemmArgs {
     // producer-side transform of u8_out (mode NONE = off)
     int next_mode, next_rnd;
     XformDev next_xf;
+    // residual input of the epilogue (nullptr = none)
+    const uint8_t *residual;
+    float residual_scale;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------
@@ -284,6 +287,8 @@ struct EpiView {
     int next_mode;    // SPARQ mode applied to the requantized bytes (producer-side transform)
     int next_rnd;
     XformDev next_xf;
+    const uint8_t *residual;   // u8 identity tensor added before the ReLU, or nullptr
+    float residual_scale;
 };
 
 template <class Args>
@@ -307,6 +312,8 @@ __device__ __forceinline__ EpiView make_epi_view(const Args &g)
     e.next_mode = g.next_mode;
     e.next_rnd = g.next_rnd;
     e.next_xf = g.next_xf;
+    e.residual = g.residual;
+    e.residual_scale = g.residual_scale;
     return e;
 }
 
@@ -329,21 +336,44 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[32], i
         }
     }
     if (!e.need_f) return;
+    // with a residual input the ReLU comes after the sum
+    const int relu_first = e.residual ? 0 : (int)e.relu_op;
     // v[i] becomes the fp32 value's bits in place
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
         const float4 sc = *reinterpret_cast<const float4 *>(&s_scale[ct + 4 * q]);
         const float4 bi = *reinterpret_cast<const float4 *>(&s_bias[ct + 4 * q]);
         if (e.small_acc) {
-            v[4 * q + 0] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 0], sc.x, bi.x, e.relu_op));
-            v[4 * q + 1] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 1], sc.y, bi.y, e.relu_op));
-            v[4 * q + 2] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 2], sc.z, bi.z, e.relu_op));
-            v[4 * q + 3] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 3], sc.w, bi.w, e.relu_op));
+            v[4 * q + 0] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 0], sc.x, bi.x, relu_first));
+            v[4 * q + 1] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 1], sc.y, bi.y, relu_first));
+            v[4 * q + 2] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 2], sc.z, bi.z, relu_first));
+            v[4 * q + 3] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 3], sc.w, bi.w, relu_first));
         } else {
-            v[4 * q + 0] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 0], sc.x, bi.x, e.relu_op));
-            v[4 * q + 1] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 1], sc.y, bi.y, e.relu_op));
-            v[4 * q + 2] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 2], sc.z, bi.z, e.relu_op));
-            v[4 * q + 3] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 3], sc.w, bi.w, e.relu_op));
+            v[4 * q + 0] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 0], sc.x, bi.x, relu_first));
+            v[4 * q + 1] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 1], sc.y, bi.y, relu_first));
+            v[4 * q + 2] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 2], sc.z, bi.z, relu_first));
+            v[4 * q + 3] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 3], sc.w, bi.w, relu_first));
+        }
+    }
+    if (e.residual) {
+        uint32_t r[8];
+        if (full) {
+            const uint4 r0 = __ldg(reinterpret_cast<const uint4 *>(e.residual + off));
+            const uint4 r1 = __ldg(reinterpret_cast<const uint4 *>(e.residual + off) + 1);
+            r[0] = r0.x; r[1] = r0.y; r[2] = r0.z; r[3] = r0.w;
+            r[4] = r1.x; r[5] = r1.y; r[6] = r1.z; r[7] = r1.w;
+        } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) r[q] = 0u;
+            for (int i = 0; i < 32 && col0 + i < e.N; ++i)
+                r[i >> 2] |= (uint32_t)__ldg(e.residual + off + i) << (8 * (i & 3));
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const float rv = __uint2float_rn((r[i >> 2] >> (8 * (i & 3))) & 0xFFu);
+            float y = __fmaf_rn(rv, e.residual_scale, __uint_as_float(v[i]));
+            if (e.relu_op) y = fmaxf(y, 0.0f);
+            v[i] = __float_as_uint(y);
         }
     }
     if (e.f32_out) {

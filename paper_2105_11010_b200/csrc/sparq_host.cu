@@ -9,7 +9,7 @@ namespace sparq {
 namespace {
 
 constexpr int kMaxDevices = 64;
-constexpr int kSlots = 4;   // 0: input, 1: acc, 2: f32, 3: u8
+constexpr int kSlots = 5;   // 0: input, 1: acc, 2: f32, 3: u8, 4: residual input
 
 struct Staging {
     void *ptr[kSlots] = {};
@@ -72,6 +72,18 @@ int plan_outputs(const sparq_epilogue *e, size_t elems, sparq_epilogue *dev_e, O
     dev_e->acc_out = (int32_t *)plan->dev[0];
     dev_e->f32_out = (float *)plan->dev[1];
     dev_e->u8_out = (uint8_t *)plan->dev[2];
+    return SPARQ_OK;
+}
+
+// Stages the HOST residual tensor of `e` (if any) on the device and points dev_e at the copy.
+int stage_residual(const sparq_epilogue *e, size_t elems, sparq_epilogue *dev_e, cudaStream_t st)
+{
+    if (!e->residual) return SPARQ_OK;
+    void *d = nullptr;
+    int rc = staging(4, elems, &d);
+    if (rc != SPARQ_OK) return rc;
+    if ((rc = copy(d, e->residual, elems, cudaMemcpyHostToDevice, st)) != SPARQ_OK) return rc;
+    dev_e->residual = (const uint8_t *)d;
     return SPARQ_OK;
 }
 
@@ -146,6 +158,7 @@ extern "C" int sparq_gemm_s8_host(const uint8_t *A_host, int64_t lda, const int8
     sparq_epilogue de;
     OutPlan plan;
     if ((rc = plan_outputs(e, (size_t)M * (size_t)N, &de, &plan)) != SPARQ_OK) return rc;
+    if ((rc = stage_residual(e, (size_t)M * (size_t)N, &de, st)) != SPARQ_OK) return rc;
     if ((rc = copy(d_a, A_host, (size_t)M * (size_t)lda, cudaMemcpyHostToDevice, st)) != SPARQ_OK) return rc;
     if ((rc = sparq_gemm_s8((const uint8_t *)d_a, lda, B, ldb, M, N, K, p, &de, stream)) != SPARQ_OK) return rc;
     return copy_back_and_sync(plan, st);
@@ -173,6 +186,7 @@ extern "C" int sparq_conv2d_nhwc_s8_host(const uint8_t *x_host, int n, int h, in
     sparq_epilogue de;
     OutPlan plan;
     if ((rc = plan_outputs(e, out_elems, &de, &plan)) != SPARQ_OK) return rc;
+    if ((rc = stage_residual(e, out_elems, &de, st)) != SPARQ_OK) return rc;
     if ((rc = copy(d_x, x_host, in_bytes, cudaMemcpyHostToDevice, st)) != SPARQ_OK) return rc;
     rc = sparq_conv2d_nhwc_s8((const uint8_t *)d_x, n, h, w, c, wgt, cout, r, s, stride_h, stride_w, pad_h, pad_w,
                               p, &de, stream);
