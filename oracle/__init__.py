@@ -51,6 +51,17 @@ def lib() -> ctypes.CDLL:
         L.oracle_vsparq_pair.restype = None
         L.oracle_transform.argtypes = [p, p, sz, sz, i, i, u, i]
         L.oracle_transform.restype = None
+        L.oracle_pair_fields.argtypes = [u, u, i, u, i, ctypes.POINTER(u), ctypes.POINTER(i),
+                                         ctypes.POINTER(u), ctypes.POINTER(i), ctypes.POINTER(i)]
+        L.oracle_pair_fields.restype = None
+        L.oracle_pack_states.argtypes = [i, u]
+        L.oracle_pack_states.restype = i
+        L.oracle_pack_ctrl_bits.argtypes = [i, u]
+        L.oracle_pack_ctrl_bits.restype = i
+        L.oracle_pack.argtypes = [p, sz, sz, i, u, i, p, p]
+        L.oracle_pack.restype = i
+        L.oracle_unpack.argtypes = [p, p, sz, sz, i, u, p]
+        L.oracle_unpack.restype = i
         L.oracle_gemm.argtypes = [p, p, p, i64, i64, i64, i, i, u, i]
         L.oracle_gemm.restype = None
         L.oracle_gemm_i64.argtypes = [p, p, p, i64, i64, i64, i, i, u, i]
@@ -108,6 +119,48 @@ def transform(x: np.ndarray, mode: int, n: int, mask: int, rnd: int) -> np.ndarr
     rows = x.size // row_len if row_len else 0
     if x.size:
         lib().oracle_transform(_ptr(x), _ptr(out), rows, row_len, mode, n, mask, rnd)
+    return out
+
+
+# ---- encoded form (Eq. 4, n = 4) -----------------------------------------------
+
+def pair_fields(a: int, b: int, mode: int, mask: int, rnd: int) -> Tuple[int, int, int, int, int]:
+    """(in1, opt1, in2, opt2, mux) that the multiplier of Eq. 4 receives for the pair."""
+    in1, in2 = ctypes.c_uint(0), ctypes.c_uint(0)
+    o1, o2, mux = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int(0)
+    lib().oracle_pair_fields(a, b, mode, mask, rnd, ctypes.byref(in1), ctypes.byref(o1),
+                             ctypes.byref(in2), ctypes.byref(o2), ctypes.byref(mux))
+    return int(in1.value), int(o1.value), int(in2.value), int(o2.value), int(mux.value)
+
+
+def pack_states(mode: int, mask: int) -> int:
+    return lib().oracle_pack_states(mode, mask)
+
+
+def pack_ctrl_bits(mode: int, mask: int) -> int:
+    return lib().oracle_pack_ctrl_bits(mode, mask)
+
+
+def pack(x: np.ndarray, mode: int, mask: int, rnd: int) -> Tuple[np.ndarray, np.ndarray]:
+    """(data plane, control plane) of the packed stream; rows are the last axis."""
+    x = _c(x, np.uint8)
+    row_len = x.shape[-1]
+    rows = x.size // row_len if row_len else 0
+    cb = pack_ctrl_bits(mode, mask)
+    data = np.empty(x.size // 2, dtype=np.uint8)
+    ctrl = np.empty(x.size // 16 * cb, dtype=np.uint8)
+    if lib().oracle_pack(_ptr(x), rows, row_len, mode, mask, rnd, _ptr(data), _ptr(ctrl)) != 0:
+        raise ValueError("row length must be a multiple of 16")
+    return data, ctrl
+
+
+def unpack(data: np.ndarray, ctrl: np.ndarray, shape, mode: int, mask: int) -> np.ndarray:
+    data, ctrl = _c(data, np.uint8), _c(ctrl, np.uint8)
+    out = np.empty(shape, dtype=np.uint8)
+    row_len = out.shape[-1]
+    rows = out.size // row_len if row_len else 0
+    if lib().oracle_unpack(_ptr(data), _ptr(ctrl), rows, row_len, mode, mask, _ptr(out)) != 0:
+        raise ValueError("row length must be a multiple of 16")
     return out
 
 

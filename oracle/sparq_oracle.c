@@ -146,6 +146,114 @@ void oracle_transform(const uint8_t *in, uint8_t *out, size_t rows, size_t row_l
     }
 }
 
+/* ---- Eq. 4 / Section 3.1: the encoded form -------------------------------- */
+
+/* What the multiplier of Eq. 4 receives for one pair (n = 4): two 4-bit inputs, their
+ * shift-left amounts (ShiftCtrl, "opt" in Eq. 4; the 3-bit identifier of Section 3.1 for
+ * five placements) and which weight each multiplier takes (MuxCtrl, Section 5.1):
+ *   mux 0  in1 meets the first weight, in2 the second (both activations non-zero: each
+ *          is its bSPARQ window at its own placement);
+ *   mux 1  both meet the FIRST weight: the second activation is zero and the first is
+ *          passed whole as its two nibbles, shifts 4 and 0 (Eq. 3);
+ *   mux 2  both meet the SECOND weight, same with the roles swapped.
+ * Without vSPARQ (mode 1) every pair is mux 0.  The placement stored for a window is the
+ * one of the RESULT (after rounding may have carried into the next window). */
+void oracle_pair_fields(unsigned a, unsigned b, int mode, unsigned mask, int rnd,
+                        unsigned *in1, int *opt1, unsigned *in2, int *opt2, int *mux)
+{
+    a &= 0xFFu; b &= 0xFFu;
+    if (mode == 2 && b == 0)      { *in1 = a >> 4; *opt1 = 4; *in2 = a & 15u; *opt2 = 0; *mux = 1; }
+    else if (mode == 2 && a == 0) { *in1 = b >> 4; *opt1 = 4; *in2 = b & 15u; *opt2 = 0; *mux = 2; }
+    else {
+        *in1 = oracle_bsparq_window(a, 4, mask, rnd, opt1);
+        *in2 = oracle_bsparq_window(b, 4, mask, rnd, opt2);
+        *mux = 0;
+    }
+}
+
+/* Number of allowed placements below shift s = the identifier stored for shift s. */
+static int shift_rank(int s, unsigned mask)
+{
+    int r = 0;
+    for (int t = 0; t < s; ++t) r += (int)((mask >> t) & 1u);
+    return r;
+}
+
+static int set_size(unsigned mask) { return shift_rank(5, mask); }
+
+/* The pair's metadata as ONE number ("grouping the metadata for several activations",
+ * Section 5.1, is left open by the paper; this library groups the two ShiftCtrl fields and
+ * the MuxCtrl of a pair): with ns allowed placements,
+ *   mux 0 -> id(opt1) * ns + id(opt2)      mux 1 -> ns*ns      mux 2 -> ns*ns + 1
+ * so a pair has ns*ns + 2 states with vSPARQ and ns*ns without. */
+int oracle_pack_states(int mode, unsigned mask)
+{
+    int ns = set_size(mask);
+    return ns * ns + (mode == 2 ? 2 : 0);
+}
+
+int oracle_pack_ctrl_bits(int mode, unsigned mask)
+{
+    int states = oracle_pack_states(mode, mask), bits = 0;
+    while ((1 << bits) < states) ++bits;
+    return bits;
+}
+
+/* Packed stream of `rows` rows of `row_len` activations (row_len a multiple of 16, n = 4).
+ * data: one byte per pair, (in1 << 4) | in2, pairs in order: rows * row_len / 2 bytes.
+ * ctrl: per unit of 16 activations (8 pairs) the 8 state numbers, pair j at bits
+ *       [j*cb, (j+1)*cb) of a little-endian integer of cb = ctrl_bits bytes (8 * cb bits):
+ *       rows * row_len / 16 * cb bytes.
+ * Returns 0, or -1 for an unsupported row length. */
+int oracle_pack(const uint8_t *in, size_t rows, size_t row_len, int mode, unsigned mask, int rnd,
+                uint8_t *data, uint8_t *ctrl)
+{
+    if (row_len % 16) return -1;
+    const int ns = set_size(mask), cb = oracle_pack_ctrl_bits(mode, mask);
+    for (size_t u = 0; u < rows * row_len / 16; ++u) {
+        uint64_t word = 0;
+        for (int j = 0; j < 8; ++j) {
+            unsigned in1, in2;
+            int opt1, opt2, mux;
+            oracle_pair_fields(in[16 * u + 2 * j], in[16 * u + 2 * j + 1], mode, mask, rnd,
+                               &in1, &opt1, &in2, &opt2, &mux);
+            data[8 * u + j] = (uint8_t)((in1 << 4) | in2);
+            unsigned state = mux == 0 ? (unsigned)(shift_rank(opt1, mask) * ns + shift_rank(opt2, mask))
+                                      : (unsigned)(ns * ns + mux - 1);
+            word |= (uint64_t)state << (j * cb);
+        }
+        for (int k = 0; k < cb; ++k) ctrl[(size_t)cb * u + k] = (uint8_t)(word >> (8 * k));
+    }
+    return 0;
+}
+
+/* The transformed activations T(x) back from the packed stream: Eq. 4 with unit weights,
+ * 2^opt1 * in1 and 2^opt2 * in2, routed to the pair's slots by the mux state. */
+int oracle_unpack(const uint8_t *data, const uint8_t *ctrl, size_t rows, size_t row_len,
+                  int mode, unsigned mask, uint8_t *out)
+{
+    if (row_len % 16) return -1;
+    const int ns = set_size(mask), cb = oracle_pack_ctrl_bits(mode, mask);
+    int shift_of[8], r = 0;
+    for (int t = 0; t <= 4; ++t) if ((mask >> t) & 1u) shift_of[r++] = t;
+    for (size_t u = 0; u < rows * row_len / 16; ++u) {
+        uint64_t word = 0;
+        for (int k = 0; k < cb; ++k) word |= (uint64_t)ctrl[(size_t)cb * u + k] << (8 * k);
+        for (int j = 0; j < 8; ++j) {
+            unsigned state = (unsigned)((word >> (j * cb)) & ((1u << cb) - 1u));
+            unsigned d = data[8 * u + j], qa, qb;
+            if (state < (unsigned)(ns * ns)) {
+                qa = (d >> 4) << shift_of[state / ns];
+                qb = (d & 15u) << shift_of[state % ns];
+            } else if (state == (unsigned)(ns * ns)) { qa = d; qb = 0; }
+            else { qa = 0; qb = d; }
+            out[16 * u + 2 * j] = (uint8_t)qa;
+            out[16 * u + 2 * j + 1] = (uint8_t)qb;
+        }
+    }
+    return 0;
+}
+
 /* ---- Eq. 1: the dot product over the transformed activations ------------- */
 
 /* acc[m][j] = sum_k T(A)[m][k] * B[k][j]; A is M x K (row-major, u8), B is the
