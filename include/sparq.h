@@ -208,6 +208,42 @@ SPARQ_API int sparq_gemm_s8_static(const uint8_t *A, int64_t lda, const int8_t *
                          int64_t M, int64_t N, int64_t K,
                          const sparq_params *p, const sparq_epilogue *e, void *stream);
 
+/* ---- Packed stream ------------------------------------------------------------------------
+ * The encoded form that the multiplier of Eq. 4 consumes, as a storage / bandwidth format
+ * for activations between layers (the paper names the metadata as the method's footprint
+ * cost and leaves grouping it open, Sections 5.1 and 6).  Defined for window_bits = 4 and
+ * mode BSPARQ or VSPARQ (else SPARQ_ERR_INVALID_ARG / SPARQ_ERR_UNSUPPORTED); row_len must
+ * be a multiple of 16 and all pointers 16-byte aligned (else SPARQ_ERR_UNSUPPORTED).
+ *
+ * A pair (2j, 2j+1) of a row becomes
+ *   one data byte  (in1 << 4) | in2: the two 4-bit windows of bSPARQ(a), bSPARQ(b) when the
+ *                  pair is multiplied as two windows, or the lone non-zero activation whole
+ *                  (its two nibbles, Eq. 3) when vSPARQ finds its partner zero;
+ *   one state      id(shift1) * ns + id(shift2) for two windows, where ns is the number of
+ *                  placements in the set and id(s) the rank of shift s in it (the ShiftCtrl
+ *                  fields); ns*ns when the second slot is zero; ns*ns + 1 when the first is
+ *                  (the MuxCtrl states; VSPARQ only).  The placement of a window is the
+ *                  lowest allowed one that holds the trimmed / rounded value.
+ * States take cb = sparq_packed_ctrl_bits(p) bits: 5 / 4 / 3 for 5opt / 3opt / 2opt with
+ * VSPARQ, i.e. 6.5 / 6 / 5.5 bits per activation instead of 8.
+ *   data plane: rows * row_len / 2 bytes, pairs in order.
+ *   ctrl plane: rows * row_len / 16 * cb bytes: per 16 activations the 8 states, pair j at
+ *               bits [j*cb, (j+1)*cb) of a little-endian integer of cb bytes.
+ * sparq_unpack returns T(x) exactly (what sparq_quantize writes), so a consumer may run
+ * with mode NONE on the unpacked tensor.  rows == 0 or row_len == 0 is a no-op. */
+
+/* Control bits per pair (2..5), or a negative sparq_status. */
+SPARQ_API int sparq_packed_ctrl_bits(const sparq_params *p);
+
+/* in: rows x row_len activations.  data, ctrl: the two planes (sizes above), caller-owned. */
+SPARQ_API int sparq_pack(const uint8_t *in, size_t rows, size_t row_len, const sparq_params *p,
+               uint8_t *data, uint8_t *ctrl, void *stream);
+
+/* out: rows x row_len bytes = T(x).  p must be the parameters the stream was packed with
+ * (the rounding field is ignored). */
+SPARQ_API int sparq_unpack(const uint8_t *data, const uint8_t *ctrl, size_t rows, size_t row_len,
+                 const sparq_params *p, uint8_t *out, void *stream);
+
 /* Synchronizes `stream` and reports what the device-side code recorded since the last
  * check: SPARQ_OK, SPARQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up (its
  * outputs are then undefined), or SPARQ_ERR_CUDA if the stream is in error. */

@@ -78,6 +78,12 @@ def load_library() -> ctypes.CDLL:
                                            i32, i32, i32, i32,
                                            ctypes.POINTER(_CParams), ctypes.POINTER(_CEpilogue), vp]
         L.sparq_conv2d_nhwc_s8.restype = i32
+        L.sparq_packed_ctrl_bits.argtypes = [ctypes.POINTER(_CParams)]
+        L.sparq_packed_ctrl_bits.restype = i32
+        L.sparq_pack.argtypes = [vp, sz, sz, ctypes.POINTER(_CParams), vp, vp, vp]
+        L.sparq_pack.restype = i32
+        L.sparq_unpack.argtypes = [vp, vp, sz, sz, ctypes.POINTER(_CParams), vp, vp]
+        L.sparq_unpack.restype = i32
         L.sparq_quantize_host.argtypes = L.sparq_quantize.argtypes
         L.sparq_quantize_host.restype = i32
         L.sparq_gemm_s8_host.argtypes = L.sparq_gemm_s8.argtypes
@@ -210,6 +216,47 @@ def sparq_conv2d_nhwc_s8(x: torch.Tensor, w: torch.Tensor, stride, pad, params: 
                                                _dev(w, torch.int8, "w"), cout, r, s,
                                                stride[0], stride[1], pad[0], pad[1],
                                                ctypes.byref(p), ctypes.byref(e), _stream_ptr(stream)))
+
+
+# ---- packed stream ------------------------------------------------------------------------
+
+def sparq_packed_ctrl_bits(params: SparqParams) -> int:
+    """Control bits per pair of the packed stream for these parameters."""
+    p = params._c()
+    rc = load_library().sparq_packed_ctrl_bits(ctypes.byref(p))
+    if rc < 0:
+        _raise(rc)
+    return rc
+
+
+def _rows(t: torch.Tensor):
+    row_len = t.shape[-1] if t.dim() else 1
+    return (t.numel() // row_len if row_len else 0), row_len
+
+
+def sparq_pack(inp: torch.Tensor, params: SparqParams, data: torch.Tensor, ctrl: torch.Tensor, stream=None) -> None:
+    """Packed stream of ``inp`` (rows along the last axis) into the caller's ``data``
+    (numel / 2 bytes) and ``ctrl`` (numel / 16 * ctrl_bits bytes) planes."""
+    rows, row_len = _rows(inp)
+    cb = sparq_packed_ctrl_bits(params)
+    if data.numel() < inp.numel() // 2 or ctrl.numel() < inp.numel() // 16 * cb:
+        raise ValueError("data / ctrl plane too small")
+    p = params._c()
+    _raise(load_library().sparq_pack(_dev(inp, torch.uint8, "inp"), rows, row_len, ctypes.byref(p),
+                                     _dev(data, torch.uint8, "data"), _dev(ctrl, torch.uint8, "ctrl"),
+                                     _stream_ptr(stream)))
+
+
+def sparq_unpack(data: torch.Tensor, ctrl: torch.Tensor, params: SparqParams, out: torch.Tensor, stream=None) -> None:
+    """``out`` (rows along the last axis) = T(x) of the packed stream."""
+    rows, row_len = _rows(out)
+    cb = sparq_packed_ctrl_bits(params)
+    if data.numel() < out.numel() // 2 or ctrl.numel() < out.numel() // 16 * cb:
+        raise ValueError("data / ctrl plane too small")
+    p = params._c()
+    _raise(load_library().sparq_unpack(_dev(data, torch.uint8, "data"), _dev(ctrl, torch.uint8, "ctrl"),
+                                       rows, row_len, ctypes.byref(p), _dev(out, torch.uint8, "out"),
+                                       _stream_ptr(stream)))
 
 
 # ---- host-buffer forms ------------------------------------------------------------------

@@ -21,7 +21,7 @@ def dev(a):
 
 @pytest.mark.parametrize("shape", [(300, 64, 192), (1000, 200, 128), (129, 512, 64), (257, 36, 80)])
 @pytest.mark.parametrize("relu", [False, True])
-@pytest.mark.parametrize("params", [VS, sparq.SparqParams()])
+@pytest.mark.parametrize("params", [VS, sparq.SparqParams(sparq.MODE_NONE)])
 def test_gemm_residual(shape, relu, params):
     M, N, K = shape
     A = synth.activations(M, (M, K), 0.5)
