@@ -167,6 +167,38 @@ def transform_section(device, pk, n, steps, warmup):
     return tr
 
 
+def pack_section(device, pk, n, steps, warmup):
+    """Packed stream codec on n uint8 activations (50 % zeros, rows of 1024), vSPARQ n = 4,
+    five placements, round to nearest.  Algorithmic bytes of either direction = n (raw or
+    unpacked activations) + n/2 (data plane) + n/16 * ctrl_bits (control plane)."""
+    import torch
+    import paper_2105_11010_b200 as sparq
+    sync = torch.cuda.synchronize
+    gen = torch.Generator(device=device).manual_seed(6)
+    z = torch.randn(n, generator=gen, device=device)
+    x = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
+    x[torch.rand(n, generator=gen, device=device) < 0.5] = 0
+    del z
+    x = x.view(-1, 1024)
+    p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+    cb = sparq.sparq_packed_ctrl_bits(p)
+    data = torch.empty(n // 2, dtype=torch.uint8, device=device)
+    ctrl = torch.empty(n // 16 * cb, dtype=torch.uint8, device=device)
+    y = torch.empty_like(x)
+    nbytes = n + n // 2 + n // 16 * cb
+    out = {"activations": n, "ctrl_bits_per_pair": cb, "bits_per_activation": 4 + cb / 2}
+    for name, fn in (("pack", lambda i: sparq.sparq_pack(x, p, data, ctrl)),
+                     ("unpack", lambda i: sparq.sparq_unpack(data, ctrl, p, y))):
+        ms = time_region(fn, steps, warmup, sync) / steps
+        gbs = nbytes / ms / 1e6
+        out[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1),
+                     "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
+                                  "frac": round(gbs / pk["hbm"], 4), "traffic": None,
+                                  "peak_source": pk["source"] + " copy"}}
+    sparq.sparq_check()
+    return out
+
+
 def extras(device, pk, steps):
     """Other workloads of the same library, each with its own roofline: the standalone
     transform on 2^30 activations and the ResNet-50 layer sweep at batch 64."""
@@ -175,6 +207,7 @@ def extras(device, pk, steps):
     out = {}
     sync = torch.cuda.synchronize
     out["transform_2p30"] = transform_section(device, pk, 1 << 30, 20, 3)
+    out["packed_stream_2p28"] = pack_section(device, pk, 1 << 28, 20, 3)
     # --- ResNet-50 sweep, batch 64, every conv shape (22 shapes, 52 instances) ---
     p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
     layers, total_ms, total_ops = [], 0.0, 0
@@ -282,7 +315,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the transform and ResNet-50 sweep sections")
-    ap.add_argument("--section", default="main", choices=["main", "transform"],
+    ap.add_argument("--section", default="main", choices=["main", "transform", "pack"],
                     help="'transform' times only the standalone transform kernel (small, for profiling)")
     ap.add_argument("--log2n", type=int, default=28, help="activations for --section transform (2^log2n)")
     args = ap.parse_args()
@@ -317,6 +350,9 @@ def main():
     pk = peaks()
     if args.section == "transform":
         print(json.dumps(transform_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
+        return
+    if args.section == "pack":
+        print(json.dumps(pack_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
         return
     sets = 20   # 20 x (6.4 MB in + 6.4 MB out) = 257 MB > 126 MB of L2
     xs, outs, wt, scale, bias = build_layer(device, sets)
