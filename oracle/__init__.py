@@ -72,6 +72,12 @@ def lib() -> ctypes.CDLL:
         L.oracle_epilogue.restype = None
         L.oracle_epilogue_residual.argtypes = [p, i64, i64, p, p, p, f32, i, f32, p, p]
         L.oracle_epilogue_residual.restype = None
+        L.oracle_absmax.argtypes = [p, i, sz]
+        L.oracle_absmax.restype = f32
+        L.oracle_quantize_act.argtypes = [p, i, sz, f32, p]
+        L.oracle_quantize_act.restype = None
+        L.oracle_quantize_weight.argtypes = [p, i64, i64, p, p]
+        L.oracle_quantize_weight.restype = None
         L.oracle_num_threads.restype = i
         L.oracle_set_num_threads.argtypes = [i]
         _lib = L
@@ -234,6 +240,40 @@ def epilogue(acc: np.ndarray, scale: np.ndarray, bias: Optional[np.ndarray], rel
                                        ctypes.c_float(residual_scale), int(bool(relu)),
                                        ctypes.c_float(inv_out_scale), _ptr(f), _ptr(q))
     return f, q
+
+
+# ---- uniform min-max quantization (Section 5) ---------------------------------
+
+def _fp(x: np.ndarray):
+    """(contiguous array, is_bf16): float32 arrays as they are, uint16 arrays as bf16 patterns."""
+    if x.dtype == np.uint16:
+        return np.ascontiguousarray(x), 1
+    return _c(x, np.float32), 0
+
+
+def absmax(x: np.ndarray) -> float:
+    x, bf = _fp(x)
+    return float(lib().oracle_absmax(_ptr(x), bf, x.size)) if x.size else 0.0
+
+
+def quantize_act(x: np.ndarray, max_value: float) -> np.ndarray:
+    x, bf = _fp(x)
+    out = np.empty(x.shape, dtype=np.uint8)
+    if x.size:
+        lib().oracle_quantize_act(_ptr(x), bf, x.size, ctypes.c_float(max_value), _ptr(out))
+    return out
+
+
+def quantize_weight(w: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """(int8 weights, per-kernel scale) of a float32 tensor whose first axis is the kernel."""
+    w = _c(w, np.float32)
+    cout = w.shape[0]
+    k = w.size // cout if cout else 0
+    q = np.empty(w.shape, dtype=np.int8)
+    sc = np.empty(cout, dtype=np.float32)
+    if w.size:
+        lib().oracle_quantize_weight(_ptr(w), cout, k, _ptr(q), _ptr(sc))
+    return q, sc
 
 
 def num_threads() -> int:

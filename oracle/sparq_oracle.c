@@ -396,6 +396,66 @@ void oracle_epilogue(const int32_t *acc, int64_t M, int64_t N,
     oracle_epilogue_residual(acc, M, N, scale, bias, NULL, 0.0f, relu, inv_out_scale, f32_out, u8_out);
 }
 
+/* ---- Section 5: uniform min-max quantization of the network's tensors ------ */
+
+/* The paper quantizes every layer "using a simple uniform min-max quantization, employing
+ * symmetric unsigned per-layer quantization for activations and symmetric signed
+ * per-kernel quantization for weights" (Section 5).  The statistic of both is the largest
+ * magnitude; NaNs are skipped.  bf16 inputs are given as their 16-bit patterns and widened
+ * exactly (bf16 is the top half of an fp32). */
+static float load_elem(const void *x, int is_bf16, size_t i)
+{
+    if (!is_bf16) return ((const float *)x)[i];
+    uint32_t bits = (uint32_t)((const uint16_t *)x)[i] << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return f;
+}
+
+float oracle_absmax(const void *x, int is_bf16, size_t n)
+{
+    float m = 0.0f;
+    for (size_t i = 0; i < n; ++i) {
+        float a = fabsf(load_elem(x, is_bf16, i));
+        if (a > m) m = a;                    /* false for NaN */
+    }
+    return m;
+}
+
+/* Activations, unsigned symmetric per layer: the 8-bit grid spans [0, max], so one step is
+ * max / 255.  fp32, one IEEE operation per line:
+ *     inv = 255 / max                 (0 when max is 0)
+ *     z   = x * inv
+ *     q   = clamp(rint(z), 0, 255)    nearest even; negatives and NaN -> 0 */
+void oracle_quantize_act(const void *x, int is_bf16, size_t n, float max, uint8_t *out)
+{
+    volatile float inv = max > 0.0f ? 255.0f / max : 0.0f;
+    for (size_t i = 0; i < n; ++i) {
+        volatile float z = load_elem(x, is_bf16, i) * inv;
+        volatile float u = rintf(z);
+        out[i] = !(u > 0.0f) ? 0 : u > 255.0f ? 255 : (uint8_t)u;
+    }
+}
+
+/* Weights, signed symmetric per kernel (output channel): row j of the cout x k matrix has
+ * its own largest magnitude a_j; the grid is [-127, 127] with step a_j / 127:
+ *     inv_j = 127 / a_j  (0 when a_j is 0);  q = clamp(rint(w * inv_j), -127, 127)
+ * scale_out[j] = a_j / 127 is the factor that maps the integers back. */
+void oracle_quantize_weight(const float *w, int64_t cout, int64_t k, int8_t *out, float *scale_out)
+{
+    for (int64_t j = 0; j < cout; ++j) {
+        float a = oracle_absmax(w + j * k, 0, (size_t)k);
+        volatile float inv = a > 0.0f ? 127.0f / a : 0.0f;
+        for (int64_t i = 0; i < k; ++i) {
+            volatile float z = w[j * k + i] * inv;
+            volatile float u = rintf(z);
+            out[j * k + i] = u > 127.0f ? 127 : u < -127.0f ? -127 : (u == u ? (int8_t)u : 0);
+        }
+        volatile float sc = a / 127.0f;
+        scale_out[j] = sc;
+    }
+}
+
 int oracle_num_threads(void)
 {
 #ifdef _OPENMP
