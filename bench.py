@@ -199,6 +199,31 @@ def pack_section(device, pk, n, steps, warmup):
     return out
 
 
+def frontend_section(device, pk, n, steps, warmup):
+    """Min-max quantization front end on n activations (post-ReLU normal, fp32 and bf16):
+    absmax (bytes = the input read once) and u8 quantization (input read + n bytes written)."""
+    import torch
+    import paper_2105_11010_b200 as sparq
+    sync = torch.cuda.synchronize
+    gen = torch.Generator(device=device).manual_seed(7)
+    x32 = torch.randn(n, generator=gen, device=device).clamp_(min=0)
+    out = torch.empty(n, dtype=torch.uint8, device=device)
+    mx = torch.zeros(1, dtype=torch.float32, device=device)
+    res = {"activations": n}
+    for name, x in (("f32", x32), ("bf16", x32.to(torch.bfloat16))):
+        eb = x.element_size()
+        for op, fn, nbytes in (("absmax", lambda i: sparq.sparq_absmax(x, mx), n * eb),
+                               ("quantize_u8", lambda i: sparq.sparq_quantize_act_u8(x, mx, out), n * eb + n)):
+            ms = time_region(fn, steps, warmup, sync) / steps
+            gbs = nbytes / ms / 1e6
+            res[f"{op}_{name}"] = {"ms": round(ms, 4), "gbs": round(gbs, 1),
+                                   "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"],
+                                                "unit": "GB/s", "frac": round(gbs / pk["hbm"], 4), "traffic": None,
+                                                "peak_source": pk["source"] + " copy"}}
+    sparq.sparq_check()
+    return res
+
+
 def extras(device, pk, steps):
     """Other workloads of the same library, each with its own roofline: the standalone
     transform on 2^30 activations and the ResNet-50 layer sweep at batch 64."""
@@ -208,6 +233,7 @@ def extras(device, pk, steps):
     sync = torch.cuda.synchronize
     out["transform_2p30"] = transform_section(device, pk, 1 << 30, 20, 3)
     out["packed_stream_2p28"] = pack_section(device, pk, 1 << 28, 20, 3)
+    out["minmax_frontend_2p28"] = frontend_section(device, pk, 1 << 28, 20, 3)
     # --- ResNet-50 sweep, batch 64, every conv shape (22 shapes, 52 instances) ---
     p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
     layers, total_ms, total_ops = [], 0.0, 0
@@ -315,7 +341,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the transform and ResNet-50 sweep sections")
-    ap.add_argument("--section", default="main", choices=["main", "transform", "pack"],
+    ap.add_argument("--section", default="main", choices=["main", "transform", "pack", "frontend"],
                     help="'transform' times only the standalone transform kernel (small, for profiling)")
     ap.add_argument("--log2n", type=int, default=28, help="activations for --section transform (2^log2n)")
     args = ap.parse_args()
@@ -350,6 +376,9 @@ def main():
     pk = peaks()
     if args.section == "transform":
         print(json.dumps(transform_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
+        return
+    if args.section == "frontend":
+        print(json.dumps(frontend_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
         return
     if args.section == "pack":
         print(json.dumps(pack_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))

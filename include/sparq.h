@@ -244,6 +244,35 @@ SPARQ_API int sparq_pack(const uint8_t *in, size_t rows, size_t row_len, const s
 SPARQ_API int sparq_unpack(const uint8_t *data, const uint8_t *ctrl, size_t rows, size_t row_len,
                  const sparq_params *p, uint8_t *out, void *stream);
 
+/* ---- Uniform min-max quantization (Section 5) ----------------------------------------------
+ * The paper's models are quantized "using a simple uniform min-max quantization": unsigned
+ * symmetric per layer for activations, signed symmetric per kernel for weights, with the
+ * statistics gathered over a few calibration batches.  These three calls are that front
+ * end on the device; the data set and the calibration run are the caller's.
+ * x is fp32 (SPARQ_DTYPE_F32) or bf16 (SPARQ_DTYPE_BF16, widened exactly), 16-byte aligned,
+ * any length.  fp32 arithmetic, one IEEE operation per step, as written below. */
+#define SPARQ_DTYPE_F32 0
+#define SPARQ_DTYPE_BF16 1
+
+/* *max_inout = max(*max_inout, max_i |x[i]|), NaNs skipped: a running maximum on the DEVICE
+ * (4-byte aligned), so calibration batches fold into it with no host round trip.  The
+ * caller sets it to 0 before the first batch.  n == 0 is a no-op. */
+SPARQ_API int sparq_absmax(const void *x, int dtype, size_t n, float *max_inout, void *stream);
+
+/* out[i] = clamp(rint(x[i] * inv), 0, 255) with inv = 255 / *max_dev (0 if *max_dev is 0);
+ * rint is to nearest even; negatives and NaN give 0.  max_dev is a DEVICE pointer (the
+ * statistic sparq_absmax gathered); the layer's activation scale is *max_dev / 255.
+ * out: n bytes, 16-byte aligned. */
+SPARQ_API int sparq_quantize_act_u8(const void *x, int dtype, size_t n, const float *max_dev, uint8_t *out,
+                          void *stream);
+
+/* Weights [cout][k] fp32 (k = r*s*c for a convolution): for kernel j with a_j = max |w[j][:]|,
+ * out[j][i] = clamp(rint(w[j][i] * (127 / a_j)), -127, 127) (all zero if a_j is 0; NaN -> 0)
+ * and scale_out[j] = a_j / 127.  The GEMM epilogue's scale[j] is then the activation scale
+ * times scale_out[j]. */
+SPARQ_API int sparq_quantize_weight_s8(const float *w, int64_t cout, int64_t k, int8_t *out, float *scale_out,
+                             void *stream);
+
 /* Synchronizes `stream` and reports what the device-side code recorded since the last
  * check: SPARQ_OK, SPARQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up (its
  * outputs are then undefined), or SPARQ_ERR_CUDA if the stream is in error. */

@@ -84,6 +84,12 @@ def load_library() -> ctypes.CDLL:
         L.sparq_pack.restype = i32
         L.sparq_unpack.argtypes = [vp, vp, sz, sz, ctypes.POINTER(_CParams), vp, vp]
         L.sparq_unpack.restype = i32
+        L.sparq_absmax.argtypes = [vp, i32, sz, vp, vp]
+        L.sparq_absmax.restype = i32
+        L.sparq_quantize_act_u8.argtypes = [vp, i32, sz, vp, vp, vp]
+        L.sparq_quantize_act_u8.restype = i32
+        L.sparq_quantize_weight_s8.argtypes = [vp, i64, i64, vp, vp, vp]
+        L.sparq_quantize_weight_s8.restype = i32
         L.sparq_quantize_host.argtypes = L.sparq_quantize.argtypes
         L.sparq_quantize_host.restype = i32
         L.sparq_gemm_s8_host.argtypes = L.sparq_gemm_s8.argtypes
@@ -257,6 +263,43 @@ def sparq_unpack(data: torch.Tensor, ctrl: torch.Tensor, params: SparqParams, ou
     _raise(load_library().sparq_unpack(_dev(data, torch.uint8, "data"), _dev(ctrl, torch.uint8, "ctrl"),
                                        rows, row_len, ctypes.byref(p), _dev(out, torch.uint8, "out"),
                                        _stream_ptr(stream)))
+
+
+# ---- uniform min-max quantization front end -----------------------------------------------
+
+DTYPE_F32, DTYPE_BF16 = 0, 1
+
+
+def _float_ptr(x: torch.Tensor, name: str):
+    if x is None or not x.is_cuda or not x.is_contiguous() or x.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError(f"{name} must be a contiguous CUDA tensor of float32 or bfloat16")
+    return x.data_ptr(), (DTYPE_BF16 if x.dtype == torch.bfloat16 else DTYPE_F32)
+
+
+def sparq_absmax(x: torch.Tensor, max_inout: torch.Tensor, stream=None) -> None:
+    """``max_inout[0] = max(max_inout[0], max |x|)`` on the device (float32, 1 element)."""
+    ptr, dt = _float_ptr(x, "x")
+    _raise(load_library().sparq_absmax(ptr, dt, x.numel(), _dev(max_inout, torch.float32, "max_inout"),
+                                       _stream_ptr(stream)))
+
+
+def sparq_quantize_act_u8(x: torch.Tensor, max_dev: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    """Unsigned symmetric per-layer quantization of ``x`` onto [0, max] in 255 steps."""
+    ptr, dt = _float_ptr(x, "x")
+    if out.numel() < x.numel():
+        raise ValueError("out is smaller than x")
+    _raise(load_library().sparq_quantize_act_u8(ptr, dt, x.numel(), _dev(max_dev, torch.float32, "max_dev"),
+                                                _dev(out, torch.uint8, "out"), _stream_ptr(stream)))
+
+
+def sparq_quantize_weight_s8(w: torch.Tensor, out: torch.Tensor, scale_out: torch.Tensor, stream=None) -> None:
+    """Signed symmetric per-kernel quantization of float32 ``w`` (kernels along axis 0)."""
+    cout = w.shape[0]
+    k = w.numel() // cout if cout else 0
+    if out.numel() < w.numel() or scale_out.numel() < cout:
+        raise ValueError("out / scale_out too small")
+    _raise(load_library().sparq_quantize_weight_s8(_dev(w, torch.float32, "w"), cout, k, _dev(out, torch.int8, "out"),
+                                                   _dev(scale_out, torch.float32, "scale_out"), _stream_ptr(stream)))
 
 
 # ---- host-buffer forms ------------------------------------------------------------------

@@ -85,17 +85,20 @@ __device__ __forceinline__ uint32_t lut_half(const uint8_t *s_lut, uint32_t off)
 template <int POS, int CB>
 __device__ __forceinline__ void put_state(uint32_t &lo, uint32_t &hi, uint32_t st)
 {
-    if (POS < 32) lo |= st << POS;
-    if (POS >= 32) hi |= st << (POS - 32);
-    else if (POS + CB > 32) hi |= st >> (32 - POS);
+    if constexpr (POS >= 32) {
+        hi |= st << (POS - 32);
+    } else {
+        lo |= st << POS;
+        if constexpr (POS + CB > 32) hi |= st >> (32 - POS);
+    }
 }
 
 template <int POS, int CB>
 __device__ __forceinline__ uint32_t get_state(uint32_t lo, uint32_t hi)
 {
     uint32_t v;
-    if (POS >= 32) v = hi >> (POS - 32);
-    else if (POS + CB > 32) v = __funnelshift_r(lo, hi, POS);
+    if constexpr (POS >= 32) v = hi >> (POS - 32);
+    else if constexpr (POS + CB > 32) v = __funnelshift_r(lo, hi, POS);
     else v = lo >> POS;
     return v & ((1u << CB) - 1u);
 }
