@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_unpack.restype = i
         L.oracle_gemm.argtypes = [p, p, p, i64, i64, i64, i, i, u, i]
         L.oracle_gemm.restype = None
+        L.oracle_gemm_sparse24.argtypes = [p, p, p, p, i64, i64, i64, i, i, u, i]
+        L.oracle_gemm_sparse24.restype = i
         L.oracle_gemm_i64.argtypes = [p, p, p, i64, i64, i64, i, i, u, i]
         L.oracle_gemm_i64.restype = None
         L.oracle_conv2d_nhwc.argtypes = [p, i, i, i, i, p, i, i, i, i, i, i, i, i, i, u, i, p, i64, p]
@@ -179,6 +181,20 @@ def gemm(A: np.ndarray, B: np.ndarray, mode: int, n: int, mask: int, rnd: int) -
     acc = np.zeros((M, N), dtype=np.int32)
     if acc.size:
         lib().oracle_gemm(_ptr(A), _ptr(B), _ptr(acc), M, N, K, mode, n, mask, rnd)
+    return acc
+
+
+def gemm_sparse24(A: np.ndarray, vals: np.ndarray, pos: np.ndarray, mode: int, n: int, mask: int, rnd: int) -> np.ndarray:
+    """int32 product of A (M, K) uint8 with 2:4-compressed weights: vals (N, K/2) int8 and
+    their coordinates pos (N, K/2) uint8 inside each group of four; the SPARQ pair is the
+    pair of activations the coordinates select."""
+    A, vals, pos = _c(A, np.uint8), _c(vals, np.int8), _c(pos, np.uint8)
+    M, K = A.shape
+    N = vals.shape[0]
+    assert vals.shape == (N, K // 2) and pos.shape == (N, K // 2)
+    acc = np.zeros((M, N), dtype=np.int32)
+    if acc.size and lib().oracle_gemm_sparse24(_ptr(A), _ptr(vals), _ptr(pos), _ptr(acc), M, N, K, mode, n, mask, rnd) != 0:
+        raise ValueError("K must be a multiple of 4 and coordinates strictly increasing in 0..3")
     return acc
 
 

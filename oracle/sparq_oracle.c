@@ -280,6 +280,45 @@ void oracle_gemm(const uint8_t *A, const int8_t *B, int32_t *acc,
     }
 }
 
+/* ---- Section 4 / 5.3: SPARQ on top of a sparse tensor core ------------------- */
+
+/* Weights pruned 2:4 are stored compressed: per output channel j and per group g of four
+ * consecutive reduction indices, the two kept values vals[j][2g], vals[j][2g+1] and their
+ * coordinates pos[j][2g] < pos[j][2g+1] in 0..3 (Section 4, "Only the non-zero-value
+ * weights are stored with additional coordinates").  The coordinates pick two of the
+ * group's four activations; vSPARQ then looks at THAT pair (Section 5.3: activations are
+ * "first filtered through the multiplexers ... Then, vSPARQ comes into play, inspecting
+ * pairs of activations"), so the transform depends on the output channel:
+ *     acc[m][j] = sum_g  T2(A[m][4g+p0], A[m][4g+p1]) . (v0, v1)
+ * with T2 the pair rule of Eq. 2 (mode 2), bSPARQ on each (mode 1) or the identity (mode 0).
+ * K must be a multiple of 4.  Returns 0, or -1 for bad coordinates. */
+int oracle_gemm_sparse24(const uint8_t *A, const int8_t *vals, const uint8_t *pos, int32_t *acc,
+                         int64_t M, int64_t N, int64_t K, int mode, int n, unsigned mask, int rnd)
+{
+    if (K % 4) return -1;
+    for (int64_t j = 0; j < N; ++j)
+        for (int64_t g = 0; g < K / 4; ++g) {
+            unsigned p0 = pos[j * (K / 2) + 2 * g], p1 = pos[j * (K / 2) + 2 * g + 1];
+            if (p0 >= p1 || p1 > 3) return -1;
+        }
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        for (int64_t j = 0; j < N; ++j) {
+            int32_t sum = 0;
+            for (int64_t g = 0; g < K / 4; ++g) {
+                const int64_t c = j * (K / 2) + 2 * g;
+                unsigned a = A[m * K + 4 * g + pos[c]], b = A[m * K + 4 * g + pos[c + 1]], qa, qb;
+                if (mode == 2) oracle_vsparq_pair(a, b, n, mask, rnd, &qa, &qb);
+                else if (mode == 1) { qa = oracle_bsparq(a, n, mask, rnd); qb = oracle_bsparq(b, n, mask, rnd); }
+                else { qa = a; qb = b; }
+                sum += (int32_t)qa * (int32_t)vals[c] + (int32_t)qb * (int32_t)vals[c + 1];
+            }
+            acc[m * N + j] = sum;
+        }
+    }
+    return 0;
+}
+
 /* Same product accumulated in 64 bits (tiny shapes only): equality with the int32
  * result shows that the 32-bit accumulator never wrapped. */
 void oracle_gemm_i64(const uint8_t *A, const int8_t *B, int64_t *acc,

@@ -22,4 +22,6 @@ from .generators import (  # noqa: F401
     resnet50_conv_layers,
     conv_out_hw,
     inv_out_scale,
+    sparse24_weights,
+    sparse24_dense,
 )

@@ -138,3 +138,25 @@ def inv_out_scale(k: int, zero_frac: float = 0.5) -> float:
     to 40 on the next layer's uint8 grid (the activations' own half-normal)."""
     sigma_acc = (k * (1.0 - zero_frac) * 1600.0 * 900.0) ** 0.5
     return float(np.float32(40.0 / (sigma_acc * 0.0055)))
+
+
+def sparse24_weights(seed: int, n_out: int, k: int, stream: int = 1):
+    """2:4 structured-sparse weights in compressed form: (vals (n_out, k/2) int8, pos (n_out,
+    k/2) uint8).  In every group of four reduction indices two coordinates are kept,
+    uniformly among the six choices, in increasing order; values as `weights`."""
+    assert k % 4 == 0
+    vals = weights(seed, (n_out, k // 2))
+    rng = _rng(seed, stream + 16)
+    combos = np.array([(0, 1), (0, 2), (0, 3), (1, 2), (1, 3), (2, 3)], dtype=np.uint8)
+    pick = rng.integers(0, 6, size=(n_out, k // 4))
+    pos = combos[pick].reshape(n_out, k // 2)
+    return vals, np.ascontiguousarray(pos)
+
+
+def sparse24_dense(vals: np.ndarray, pos: np.ndarray) -> np.ndarray:
+    """The dense (n_out, k) int8 matrix that the compressed form stands for (data movement only)."""
+    n_out, half = vals.shape
+    dense = np.zeros((n_out, half * 2), dtype=np.int8)
+    cols = (np.arange(half) // 2 * 4)[None, :] + pos.astype(np.int64)
+    np.put_along_axis(dense, cols, vals, axis=1)
+    return dense
