@@ -273,9 +273,46 @@ SPARQ_API int sparq_quantize_act_u8(const void *x, int dtype, size_t n, const fl
 SPARQ_API int sparq_quantize_weight_s8(const float *w, int64_t cout, int64_t k, int8_t *out, float *scale_out,
                              void *stream);
 
+/* ---- 2:4 sparse weights (Sections 4 and 5.3) ---------------------------------------------
+ * Weights pruned 2:4 arrive compressed as a sparse tensor core stores them: per output
+ * channel j and per group of four consecutive reduction indices, the two kept values
+ * vals[j][2g], vals[j][2g+1] and their coordinates pos[j][2g] < pos[j][2g+1] in 0..3.  The
+ * coordinates select two of the group's four activations, and vSPARQ then pairs THOSE two
+ * (Section 5.3), so the transform depends on the output channel:
+ *     acc[m][j] = sum_g T2(A[m][4g+p0], A[m][4g+p1]) . (v0, v1)
+ * The library computes this exactly as a dense contraction over expanded operands: the
+ * activations of a group become the six pairs a pattern could select, transformed
+ * ((0,1) (0,2) (0,3) (1,2) (1,3) (2,3): 12 bytes per 4), and a weight row holds its two
+ * values in its own pattern's two columns.  With mode NONE or BSPARQ the transform is per
+ * element and the expansion is the dense form of the weights (K' = K); with VSPARQ
+ * K' = 3K.  The expanded tensors are ordinary operands of sparq_gemm_s8 /
+ * sparq_conv2d_nhwc_s8 with mode NONE (for a convolution expand along the channel axis:
+ * rows = pixels, K = c; weights [cout][r][s][c] -> [cout][r][s][c']). */
+
+/* K' for these parameters, or a negative sparq_status (K must be a multiple of 4). */
+SPARQ_API int64_t sparq_sparse24_expanded_k(int64_t K, const sparq_params *p);
+
+/* vals [N][K/2] s8, pos [N][K/2] u8 -> w_exp [N][K'] s8 (4-byte aligned).  A group whose
+ * coordinates are not strictly increasing in 0..3 is expanded as zeros and recorded:
+ * the next sparq_check returns SPARQ_ERR_INVALID_ARG. */
+SPARQ_API int sparq_sparse24_expand_weights(const int8_t *vals, const uint8_t *pos, int64_t N, int64_t K,
+                                  const sparq_params *p, int8_t *w_exp, void *stream);
+
+/* A [rows][K] u8 -> a_exp [rows][K'] u8: the transformed candidate pairs (VSPARQ), or T(A)
+ * itself (NONE, BSPARQ).  K a multiple of 16, both pointers 16-byte aligned. */
+SPARQ_API int sparq_sparse24_expand_activations(const uint8_t *A, size_t rows, size_t K, const sparq_params *p,
+                                      uint8_t *a_exp, void *stream);
+
+/* The product above followed by the epilogue `e`.  w_exp: expanded weights for the same
+ * parameters.  workspace: M * K' bytes, 16-byte aligned, caller-owned (VSPARQ only; may be
+ * NULL otherwise).  Other requirements as for sparq_gemm_s8. */
+SPARQ_API int sparq_gemm_s8_sparse24(const uint8_t *A, const int8_t *w_exp, int64_t M, int64_t N, int64_t K,
+                           const sparq_params *p, const sparq_epilogue *e, uint8_t *workspace, void *stream);
+
 /* Synchronizes `stream` and reports what the device-side code recorded since the last
  * check: SPARQ_OK, SPARQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up (its
- * outputs are then undefined), or SPARQ_ERR_CUDA if the stream is in error. */
+ * outputs are then undefined), SPARQ_ERR_INVALID_ARG if sparq_sparse24_expand_weights met
+ * bad coordinates, or SPARQ_ERR_CUDA if the stream is in error. */
 SPARQ_API int sparq_check(void *stream);
 
 /* Text of the calling thread's most recent error ("" if none).  The pointer stays valid

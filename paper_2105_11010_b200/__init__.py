@@ -16,6 +16,8 @@ from ._binding import (  # noqa: F401
     sparq_quantize_host, sparq_gemm_s8_host, sparq_conv2d_nhwc_s8_host,
     sparq_gemm_s8_static, STATIC_SCRATCH_BYTES,
     sparq_packed_ctrl_bits, sparq_pack, sparq_unpack,
+    sparq_sparse24_expanded_k, sparq_sparse24_expand_weights, sparq_sparse24_expand_activations,
+    sparq_gemm_s8_sparse24,
     sparq_absmax, sparq_quantize_act_u8, sparq_quantize_weight_s8, DTYPE_F32, DTYPE_BF16,
     sparq_check, sparq_last_error, sparq_shutdown,
 )

@@ -90,6 +90,15 @@ def load_library() -> ctypes.CDLL:
         L.sparq_quantize_act_u8.restype = i32
         L.sparq_quantize_weight_s8.argtypes = [vp, i64, i64, vp, vp, vp]
         L.sparq_quantize_weight_s8.restype = i32
+        L.sparq_sparse24_expanded_k.argtypes = [i64, ctypes.POINTER(_CParams)]
+        L.sparq_sparse24_expanded_k.restype = i64
+        L.sparq_sparse24_expand_weights.argtypes = [vp, vp, i64, i64, ctypes.POINTER(_CParams), vp, vp]
+        L.sparq_sparse24_expand_weights.restype = i32
+        L.sparq_sparse24_expand_activations.argtypes = [vp, sz, sz, ctypes.POINTER(_CParams), vp, vp]
+        L.sparq_sparse24_expand_activations.restype = i32
+        L.sparq_gemm_s8_sparse24.argtypes = [vp, vp, i64, i64, i64, ctypes.POINTER(_CParams),
+                                             ctypes.POINTER(_CEpilogue), vp, vp]
+        L.sparq_gemm_s8_sparse24.restype = i32
         L.sparq_quantize_host.argtypes = L.sparq_quantize.argtypes
         L.sparq_quantize_host.restype = i32
         L.sparq_gemm_s8_host.argtypes = L.sparq_gemm_s8.argtypes
@@ -300,6 +309,61 @@ def sparq_quantize_weight_s8(w: torch.Tensor, out: torch.Tensor, scale_out: torc
         raise ValueError("out / scale_out too small")
     _raise(load_library().sparq_quantize_weight_s8(_dev(w, torch.float32, "w"), cout, k, _dev(out, torch.int8, "out"),
                                                    _dev(scale_out, torch.float32, "scale_out"), _stream_ptr(stream)))
+
+
+# ---- 2:4 sparse weights ---------------------------------------------------------------------
+
+def sparq_sparse24_expanded_k(K: int, params: SparqParams) -> int:
+    p = params._c()
+    rc = load_library().sparq_sparse24_expanded_k(K, ctypes.byref(p))
+    if rc < 0:
+        _raise(int(rc))
+    return int(rc)
+
+
+def sparq_sparse24_expand_weights(vals: torch.Tensor, pos: torch.Tensor, params: SparqParams, w_exp: torch.Tensor,
+                                  stream=None) -> None:
+    """Compressed 2:4 weights (vals, pos: (N, K/2)) -> ``w_exp`` (N, K')."""
+    N = vals.shape[0]
+    K = 2 * (vals.numel() // N) if N else 0
+    if pos.numel() != vals.numel() or w_exp.numel() < N * sparq_sparse24_expanded_k(K, params):
+        raise ValueError("pos / w_exp size does not match vals")
+    p = params._c()
+    _raise(load_library().sparq_sparse24_expand_weights(_dev(vals, torch.int8, "vals"), _dev(pos, torch.uint8, "pos"),
+                                                        N, K, ctypes.byref(p), _dev(w_exp, torch.int8, "w_exp"),
+                                                        _stream_ptr(stream)))
+
+
+def sparq_sparse24_expand_activations(A: torch.Tensor, params: SparqParams, a_exp: torch.Tensor, stream=None) -> None:
+    """Activations (rows along the last axis, K) -> ``a_exp`` with K' per row."""
+    rows, K = _rows(A)
+    if a_exp.numel() < rows * sparq_sparse24_expanded_k(K, params):
+        raise ValueError("a_exp too small")
+    p = params._c()
+    _raise(load_library().sparq_sparse24_expand_activations(_dev(A, torch.uint8, "A"), rows, K, ctypes.byref(p),
+                                                            _dev(a_exp, torch.uint8, "a_exp"), _stream_ptr(stream)))
+
+
+def sparq_gemm_s8_sparse24(A: torch.Tensor, w_exp: torch.Tensor, params: SparqParams, *,
+                           workspace: Optional[torch.Tensor] = None,
+                           scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                           relu: bool = False, inv_out_scale: float = 1.0,
+                           acc_out: Optional[torch.Tensor] = None, f32_out: Optional[torch.Tensor] = None,
+                           u8_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """``acc[m][j] = sum_g T2(selected pair) . (v0, v1)`` for 2:4 weights expanded by
+    :func:`sparq_sparse24_expand_weights`, then the epilogue."""
+    M, K = A.shape
+    N = w_exp.shape[0]
+    kx = sparq_sparse24_expanded_k(K, params)
+    if w_exp.numel() != N * kx:
+        raise ValueError("w_exp does not have N * K' elements")
+    if workspace is not None and workspace.numel() < M * kx:
+        raise ValueError("workspace smaller than M * K'")
+    p = params._c()
+    e = _epilogue(N, scale, bias, relu, inv_out_scale, acc_out, f32_out, u8_out)
+    _raise(load_library().sparq_gemm_s8_sparse24(_dev(A, torch.uint8, "A"), _dev(w_exp, torch.int8, "w_exp"), M, N, K,
+                                                 ctypes.byref(p), ctypes.byref(e),
+                                                 _dev(workspace, torch.uint8, "workspace"), _stream_ptr(stream)))
 
 
 # ---- host-buffer forms ------------------------------------------------------------------

@@ -122,6 +122,8 @@ extern "C" int sparq_check(void *stream)
     if (e != cudaSuccess) return cuda_error(e, "cudaMemcpy(status word)");
     if (word) {
         cudaMemset(p, 0, sizeof(word));
+        if (word == 0x100u)
+            return set_error(SPARQ_ERR_INVALID_ARG, "2:4 weight coordinates were not strictly increasing in 0..3; those groups were expanded as zeros");
         return set_error(SPARQ_ERR_TIMEOUT, "a bounded device-side wait expired (status 0x%x); outputs of the affected launch are undefined", word);
     }
     return SPARQ_OK;
