@@ -224,6 +224,43 @@ def frontend_section(device, pk, n, steps, warmup):
     return res
 
 
+def sparse24_section(device, pk, steps, warmup):
+    """vSPARQ on 2:4 sparse weights, shape of the 28x28x128 -> 128 3x3 layer at batch 128
+    (M 100352, K 1152, N 128): expansion of the activations (bytes = M*K read + 3*M*K
+    written), then the dense contraction over the expanded operands.  Ops are counted as
+    the sparse tensor core would: 2*M*N*K/2."""
+    import torch
+    import paper_2105_11010_b200 as sparq
+    sync = torch.cuda.synchronize
+    M, K, N = 100352, 1152, 128
+    p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+    gen = torch.Generator(device=device).manual_seed(8)
+    z = torch.randn(M * K, generator=gen, device=device)
+    A = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
+    A[torch.rand(M * K, generator=gen, device=device) < 0.5] = 0
+    A = A.view(M, K)
+    del z
+    vals, pos = synth.sparse24_weights(8, N, K)
+    w = torch.empty((N, 3 * K), dtype=torch.int8, device=device)
+    sparq.sparq_sparse24_expand_weights(torch.from_numpy(vals).to(device), torch.from_numpy(pos).to(device), p, w)
+    ws = torch.empty(M * 3 * K, dtype=torch.uint8, device=device)
+    sc = torch.from_numpy(synth.scales(8, N)).to(device)
+    out = torch.empty((M, N), dtype=torch.uint8, device=device)
+    inv = synth.inv_out_scale(K // 2)
+    ms_e = time_region(lambda i: sparq.sparq_sparse24_expand_activations(A, p, ws), steps, warmup, sync) / steps
+    ms_t = time_region(lambda i: sparq.sparq_gemm_s8_sparse24(A, w, p, workspace=ws, scale=sc, relu=True,
+                                                              inv_out_scale=inv, u8_out=out), steps, warmup, sync) / steps
+    sparq.sparq_check()
+    gbs = 4 * M * K / ms_e / 1e6
+    return {"shape": {"M": M, "K": K, "N": N},
+            "expand_activations": {"ms": round(ms_e, 4), "gbs": round(gbs, 1),
+                                   "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
+                                                "frac": round(gbs / pk["hbm"], 4), "traffic": None,
+                                                "peak_source": pk["source"] + " copy"}},
+            "gemm_sparse24": {"ms": round(ms_t, 4), "sparse_tops": round(M * N * K / ms_t / 1e9, 1),
+                              "dense_equivalent_tops_executed": round(2 * M * N * 3 * K / ms_t / 1e9, 1)}}
+
+
 def extras(device, pk, steps):
     """Other workloads of the same library, each with its own roofline: the standalone
     transform on 2^30 activations and the ResNet-50 layer sweep at batch 64."""
@@ -234,6 +271,7 @@ def extras(device, pk, steps):
     out["transform_2p30"] = transform_section(device, pk, 1 << 30, 20, 3)
     out["packed_stream_2p28"] = pack_section(device, pk, 1 << 28, 20, 3)
     out["minmax_frontend_2p28"] = frontend_section(device, pk, 1 << 28, 20, 3)
+    out["sparse24_vsparq"] = sparse24_section(device, pk, 20, 3)
     # --- ResNet-50 sweep, batch 64, every conv shape (22 shapes, 52 instances) ---
     p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
     layers, total_ms, total_ops = [], 0.0, 0
@@ -341,7 +379,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the transform and ResNet-50 sweep sections")
-    ap.add_argument("--section", default="main", choices=["main", "transform", "pack", "frontend"],
+    ap.add_argument("--section", default="main", choices=["main", "transform", "pack", "frontend", "sparse24"],
                     help="'transform' times only the standalone transform kernel (small, for profiling)")
     ap.add_argument("--log2n", type=int, default=28, help="activations for --section transform (2^log2n)")
     args = ap.parse_args()
@@ -376,6 +414,9 @@ def main():
     pk = peaks()
     if args.section == "transform":
         print(json.dumps(transform_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
+        return
+    if args.section == "sparse24":
+        print(json.dumps(sparse24_section(device, pk, args.steps, args.warmup)))
         return
     if args.section == "frontend":
         print(json.dumps(frontend_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
