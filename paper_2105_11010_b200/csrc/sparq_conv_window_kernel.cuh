@@ -211,7 +211,11 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         __syncwarp();
     } else if (warp == 1) {
         // ================= MMA issuer =================
-        if (lane == 0) {
+        // The whole warp runs this loop converged and one elected lane issues: the descriptor
+        // arithmetic below is on warp-uniform values only (kernel arguments, loop counters),
+        // which lets it stay in the uniform datapath that feeds tcgen05.mma.
+        {
+            const uint32_t elected = elect_one();
             constexpr uint32_t idesc = make_idesc_i8(BN);
             // descriptors of window buffer 0 and of weight slot 0; offsets are added in units of
             // 16 bytes to the start-address field (the low word never carries into the next field)
@@ -225,7 +229,14 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             constexpr int kRegTab = 18;         // 3x3 taps of up to two channel blocks
             uint2 rtab[kRegTab];
 #pragma unroll
-            for (int kb = 0; kb < kRegTab; ++kb) rtab[kb] = (kb < kb_count) ? s_tab[kb] : make_uint2(0u, 0u);
+            for (int kb = 0; kb < kRegTab; ++kb) {
+                // same entries as s_tab, from the kernel arguments
+                const int cb = kb / taps, tap = kb % taps;
+                const uint32_t rows = (uint32_t)((tap / g.S) * g.Wp + (tap % g.S));
+                rtab[kb] = (kb < kb_count) ? make_uint2(((uint32_t)cb * (uint32_t)g.plane_bytes + rows * CB) >> 4,
+                                                        (uint32_t)kb * (uint32_t)(kBBlock >> 4))
+                                           : make_uint2(0u, 0u);
+            }
             if (B_RESIDENT) SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status));
             for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
                 const int acc = wt & 1;
@@ -251,10 +262,10 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                     const uint64_t adesc = a_desc0 + (uint64_t)e.x;
 #pragma unroll
                     for (int k = 0; k < CB / 32; ++k)
-                        tc_mma_i8(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
-                                  (kb > 0 || k > 0) ? 1u : 0u);
+                        tc_mma_i8_if(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
+                                     (kb > 0 || k > 0) ? 1u : 0u, elected);
                     if (!B_RESIDENT) {
-                        tc_commit(smem_u32(&bar_b_empty[s]));
+                        tc_commit_if(smem_u32(&bar_b_empty[s]), elected);
                         if (++s == g.b_stages) { s = 0; bph ^= 1u; }
                     }
                 };
@@ -267,8 +278,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                     for (int kb = 0; kb < kb_count; ++kb) issue_block(kb, s_tab[kb]);
                 }
                 mi += SPARQ_PROF_NOW() - is0;
-                tc_commit(smem_u32(&bar_win_empty[b]));       // window reusable once these MMAs retire
-                tc_commit(smem_u32(&bar_acc_full[acc]));      // accumulator complete
+                tc_commit_if(smem_u32(&bar_win_empty[b]), elected);       // window reusable once these MMAs retire
+                tc_commit_if(smem_u32(&bar_acc_full[acc]), elected);      // accumulator complete
                 if (++b == g.win_bufs) { b = 0; wph ^= 1u; }
             }
             SPARQ_PROF_STORE(2, mw);
@@ -276,7 +287,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             SPARQ_PROF_STORE(11, mb);
             SPARQ_PROF_STORE(12, mi);
             SPARQ_PROF_STORE(4, SPARQ_PROF_NOW() - mt0);
-            tc_commit(smem_u32(&bar_done));
+            tc_commit_if(smem_u32(&bar_done), elected);
             mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, true);
         }
         __syncwarp();
@@ -296,6 +307,76 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         const bool slot_ok = (tr < g.TR) && (ow < g.Wo);
         long long ew = 0;
         const long long et0 = SPARQ_PROF_NOW();
+        // 64-wide tiles have one column tile and one 32-column chunk per warp.  When only the
+        // requantized bytes are wanted (the form every layer of a network uses), the warp keeps
+        // the scale and bias of its 32 columns in registers for the whole launch -- shared-memory
+        // reads queue behind the tensor core's operand fetches -- and takes the accumulator in
+        // two 16-column halves so that those 64 registers fit beside it.
+        if (BN == 64 && ev.need_f && !g.acc_out && !g.f32_out && !g.residual && g.N == 64) {
+            epi_stage_scale_bias(g, 0, BN, et, s_scale, s_bias);
+            const int cbase = half * 32;
+            float rs[32], rb[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                rs[i] = s_scale[cbase + i];
+                rb[i] = s_bias[cbase + i];
+            }
+            const uint32_t tiles32 = (uint32_t)total_tiles, tpi = (uint32_t)g.tiles_per_img;
+            for (uint32_t tile = blockIdx.x; tile < tiles32; tile += gridDim.x, ++wt) {
+                const uint32_t acc = wt & 1u;
+                // coordinates first: they do not depend on the accumulator
+                const uint32_t img = tile / tpi;
+                const int oh = (int)(tile - img * tpi) * g.TR + tr;
+                const bool row_ok = slot_ok && (oh < g.Ho);
+                uint8_t *dst = g.u8_out + (((int64_t)img * g.Ho + oh) * g.Wo + ow) * 64 + cbase;
+                const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + (uint32_t)cbase;
+                SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt >> 1) & 1u, abort_flag, g.status));
+                tc_fence_after();
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    uint32_t v[16];
+                    tmem_ld_32x16_issue(taddr0 + (uint32_t)(hh * 16), v);
+                    tmem_ld_wait();
+                    if (hh == 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
+                    }
+                    if (!row_ok) continue;
+                    uint32_t w[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t b[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int c = hh * 16 + 4 * q + j;
+                            const float y = ev.small_acc ? dequant<true>((int32_t)v[4 * q + j], rs[c], rb[c], ev.relu_op)
+                                                         : dequant<false>((int32_t)v[4 * q + j], rs[c], rb[c], ev.relu_op);
+                            b[j] = requant_bits(y, ev.inv_out_scale);
+                        }
+                        w[q] = pack4(b[0], b[1], b[2], b[3]);
+                    }
+                    if (ev.next_mode != SPARQ_MODE_NONE) {
+                        const bool fast4 = ev.next_xf.n == 4 && ev.next_xf.rounds == 0;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            if (ev.next_mode == SPARQ_MODE_VSPARQ) {
+                                if (fast4) w[q] = ev.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 4, true, false>(w[q], ev.next_xf)
+                                                              : xform_word<SPARQ_MODE_VSPARQ, 4, false, false>(w[q], ev.next_xf);
+                                else w[q] = ev.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 0, true, true>(w[q], ev.next_xf)
+                                                        : xform_word<SPARQ_MODE_VSPARQ, 0, false, true>(w[q], ev.next_xf);
+                            } else {
+                                if (fast4) w[q] = ev.next_rnd ? xform_word<SPARQ_MODE_BSPARQ, 4, true, false>(w[q], ev.next_xf)
+                                                              : xform_word<SPARQ_MODE_BSPARQ, 4, false, false>(w[q], ev.next_xf);
+                                else w[q] = ev.next_rnd ? xform_word<SPARQ_MODE_BSPARQ, 0, true, true>(w[q], ev.next_xf)
+                                                        : xform_word<SPARQ_MODE_BSPARQ, 0, false, true>(w[q], ev.next_xf);
+                            }
+                        }
+                    }
+                    *reinterpret_cast<uint4 *>(dst + hh * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+        } else
         for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
             const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
             const int acc = wt & 1;

@@ -191,6 +191,38 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint6
         :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// The same two instructions for a warp that runs its loop converged: every lane executes
+// the surrounding code (so that descriptor arithmetic on warp-uniform values can stay in
+// the uniform datapath) and only the lane with `elected` != 0 issues.
+__device__ __forceinline__ void tc_mma_i8_if(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate, uint32_t elected)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(elected) : "memory");
+}
+
+__device__ __forceinline__ void tc_commit_if(uint32_t bar, uint32_t elected)
+{
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        :: "r"(bar), "r"(elected) : "memory");
+}
+
+// One lane of a converged warp (the same lane every time it is asked within a launch is not
+// guaranteed; callers ask once and keep the answer).
+__device__ __forceinline__ uint32_t elect_one()
+{
+    uint32_t e;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(e));
+    return e;
+}
+
 // Shared-memory matrix descriptor of a K-major tile whose rows are ROW_BYTES long
 // (128 or 64) and swizzled with the matching TMA mode; 8-row groups are contiguous.
 template <int ROW_BYTES>
@@ -238,6 +270,16 @@ __device__ __forceinline__ void tmem_ld_32x32_issue(uint32_t taddr, uint32_t (&r
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_32x16_issue(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr) : "memory");
 }
 
@@ -317,22 +359,28 @@ __device__ __forceinline__ EpiView make_epi_view(const Args &g)
     return e;
 }
 
-// One thread's 32 consecutive accumulators of output row `row` (columns col0 .. col0+31,
-// tile-local column ct): optional raw store, dequantize, optional fp32 store, requantize
-// and store.  v is overwritten.
-__device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[32], int64_t row, int64_t col0, int ct,
-                                          const float *s_scale, const float *s_bias)
+// One thread's NV (32 or 16) consecutive accumulators of output row `row` (columns col0 ..
+// col0+NV-1, tile-local column ct): optional raw store, dequantize, optional fp32 store,
+// requantize and store.  v is overwritten.
+// REG: scale and bias of the NV columns come from the caller's registers rs / rb instead of
+// shared memory (shared-memory reads queue behind the tensor core's operand fetches).
+template <int NV = 32, bool REG = false>
+__device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[NV], int64_t row, int64_t col0, int ct,
+                                          const float *s_scale, const float *s_bias,
+                                          const float *rs = nullptr, const float *rb = nullptr)
 {
+    static_assert(NV == 32 || NV == 16, "chunk width");
+    constexpr int NQ = NV / 4;      // groups of four columns = words of packed bytes
     const int64_t off = row * e.N + col0;
-    const bool full = e.vec_ok && (col0 + 32 <= e.N);
+    const bool full = e.vec_ok && (col0 + NV <= e.N);
     if (e.acc_out) {
         if (full) {
             int4 *dst = reinterpret_cast<int4 *>(e.acc_out + off);
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
+            for (int q = 0; q < NQ; ++q)
                 dst[q] = make_int4((int)v[4 * q], (int)v[4 * q + 1], (int)v[4 * q + 2], (int)v[4 * q + 3]);
         } else {
-            for (int i = 0; i < 32 && col0 + i < e.N; ++i) e.acc_out[off + i] = (int32_t)v[i];
+            for (int i = 0; i < NV && col0 + i < e.N; ++i) e.acc_out[off + i] = (int32_t)v[i];
         }
     }
     if (!e.need_f) return;
@@ -340,9 +388,15 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[32], i
     const int relu_first = e.residual ? 0 : (int)e.relu_op;
     // v[i] becomes the fp32 value's bits in place
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-        const float4 sc = *reinterpret_cast<const float4 *>(&s_scale[ct + 4 * q]);
-        const float4 bi = *reinterpret_cast<const float4 *>(&s_bias[ct + 4 * q]);
+    for (int q = 0; q < NQ; ++q) {
+        float4 sc, bi;
+        if (REG) {
+            sc = make_float4(rs[4 * q], rs[4 * q + 1], rs[4 * q + 2], rs[4 * q + 3]);
+            bi = make_float4(rb[4 * q], rb[4 * q + 1], rb[4 * q + 2], rb[4 * q + 3]);
+        } else {
+            sc = *reinterpret_cast<const float4 *>(&s_scale[ct + 4 * q]);
+            bi = *reinterpret_cast<const float4 *>(&s_bias[ct + 4 * q]);
+        }
         if (e.small_acc) {
             v[4 * q + 0] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 0], sc.x, bi.x, relu_first));
             v[4 * q + 1] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 1], sc.y, bi.y, relu_first));
@@ -356,20 +410,21 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[32], i
         }
     }
     if (e.residual) {
-        uint32_t r[8];
+        uint32_t r[NQ];
         if (full) {
-            const uint4 r0 = __ldg(reinterpret_cast<const uint4 *>(e.residual + off));
-            const uint4 r1 = __ldg(reinterpret_cast<const uint4 *>(e.residual + off) + 1);
-            r[0] = r0.x; r[1] = r0.y; r[2] = r0.z; r[3] = r0.w;
-            r[4] = r1.x; r[5] = r1.y; r[6] = r1.z; r[7] = r1.w;
+#pragma unroll
+            for (int h = 0; h < NV / 16; ++h) {
+                const uint4 rr = __ldg(reinterpret_cast<const uint4 *>(e.residual + off) + h);
+                r[4 * h] = rr.x; r[4 * h + 1] = rr.y; r[4 * h + 2] = rr.z; r[4 * h + 3] = rr.w;
+            }
         } else {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) r[q] = 0u;
-            for (int i = 0; i < 32 && col0 + i < e.N; ++i)
+            for (int q = 0; q < NQ; ++q) r[q] = 0u;
+            for (int i = 0; i < NV && col0 + i < e.N; ++i)
                 r[i >> 2] |= (uint32_t)__ldg(e.residual + off + i) << (8 * (i & 3));
         }
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
+        for (int i = 0; i < NV; ++i) {
             const float rv = __uint2float_rn((r[i >> 2] >> (8 * (i & 3))) & 0xFFu);
             float y = __fmaf_rn(rv, e.residual_scale, __uint_as_float(v[i]));
             if (e.relu_op) y = fmaxf(y, 0.0f);
@@ -380,15 +435,15 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[32], i
         if (full) {
             uint4 *dst = reinterpret_cast<uint4 *>(e.f32_out + off);
 #pragma unroll
-            for (int q = 0; q < 8; ++q) dst[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            for (int q = 0; q < NQ; ++q) dst[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
         } else {
-            for (int i = 0; i < 32 && col0 + i < e.N; ++i) e.f32_out[off + i] = __uint_as_float(v[i]);
+            for (int i = 0; i < NV && col0 + i < e.N; ++i) e.f32_out[off + i] = __uint_as_float(v[i]);
         }
     }
     if (e.u8_out) {
-        uint32_t w[8];
+        uint32_t w[NQ];
 #pragma unroll
-        for (int q = 0; q < 8; ++q)
+        for (int q = 0; q < NQ; ++q)
             w[q] = pack4(requant_bits(__uint_as_float(v[4 * q]), e.inv_out_scale),
                          requant_bits(__uint_as_float(v[4 * q + 1]), e.inv_out_scale),
                          requant_bits(__uint_as_float(v[4 * q + 2]), e.inv_out_scale),
@@ -398,7 +453,7 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[32], i
             // channels per word, pairs (2j, 2j+1) inside it
             const bool fast4 = e.next_xf.n == 4 && e.next_xf.rounds == 0;   // n = 4, all five placements
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
+            for (int q = 0; q < NQ; ++q) {
                 if (e.next_mode == SPARQ_MODE_VSPARQ) {
                     if (fast4) w[q] = e.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 4, true, false>(w[q], e.next_xf)
                                                  : xform_word<SPARQ_MODE_VSPARQ, 4, false, false>(w[q], e.next_xf);
@@ -412,14 +467,20 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[32], i
                 }
             }
         }
-        if (full && e.u8_wide) {
-            st_global_v8(e.u8_out + off, w);
-        } else if (full) {
-            uint4 *dst = reinterpret_cast<uint4 *>(e.u8_out + off);
-            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        if (full) {
+            if constexpr (NV == 32) {
+                if (e.u8_wide) {
+                    st_global_v8(e.u8_out + off, w);
+                } else {
+                    uint4 *dst = reinterpret_cast<uint4 *>(e.u8_out + off);
+                    dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                    dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                }
+            } else {
+                *reinterpret_cast<uint4 *>(e.u8_out + off) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
         } else {
-            for (int i = 0; i < 32 && col0 + i < e.N; ++i)
+            for (int i = 0; i < NV && col0 + i < e.N; ++i)
                 e.u8_out[off + i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
         }
     }
