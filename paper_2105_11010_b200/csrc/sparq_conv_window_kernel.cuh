@@ -393,21 +393,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             const int64_t row = ((int64_t)img * g.Ho + oh) * g.Wo + ow;
             const int cbase = half * (BN / 2);
             const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + cbase);
-#pragma unroll 1
-            for (int ch = 0; ch < kChunks; ++ch) {
-                uint32_t v[32];
-                tmem_ld_32x32_issue(taddr0 + (uint32_t)(ch * 32), v);
-                tmem_ld_wait();
-                if (ch + 1 == kChunks) {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
-                }
-                const int ct = cbase + ch * 32;
-                const int64_t col0 = nt * BN + ct;
-                if (!row_ok || col0 >= g.N) continue;
-                epi_chunk(ev, v, row, col0, ct, s_scale, s_bias);
-            }
+            epi_warp_columns<kChunks>(ev, taddr0, cbase, row, row_ok, nt * BN, s_scale, s_bias,
+                                      smem_u32(&bar_acc_empty[acc]), lane);
         }
         if (warp == kFirstEpiWarp && lane == 0) {
             SPARQ_PROF_STORE(5, ew);

@@ -387,26 +387,32 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[NV], i
     // with a residual input the ReLU comes after the sum
     const int relu_first = e.residual ? 0 : (int)e.relu_op;
     // v[i] becomes the fp32 value's bits in place
+    // scale and bias of 16 columns at a time: the eight 16-byte shared-memory reads are issued
+    // together, so that their latencies (long while the tensor core is fetching operands)
+    // overlap instead of adding up
 #pragma unroll
-    for (int q = 0; q < NQ; ++q) {
-        float4 sc, bi;
-        if (REG) {
-            sc = make_float4(rs[4 * q], rs[4 * q + 1], rs[4 * q + 2], rs[4 * q + 3]);
-            bi = make_float4(rb[4 * q], rb[4 * q + 1], rb[4 * q + 2], rb[4 * q + 3]);
-        } else {
-            sc = *reinterpret_cast<const float4 *>(&s_scale[ct + 4 * q]);
-            bi = *reinterpret_cast<const float4 *>(&s_bias[ct + 4 * q]);
+    for (int h = 0; h < NV / 16; ++h) {
+        float hs[16], hb[16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (REG) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    hs[4 * q + j] = rs[16 * h + 4 * q + j];
+                    hb[4 * q + j] = rb[16 * h + 4 * q + j];
+                }
+            } else {
+                const float4 sc = *reinterpret_cast<const float4 *>(&s_scale[ct + 16 * h + 4 * q]);
+                const float4 bi = *reinterpret_cast<const float4 *>(&s_bias[ct + 16 * h + 4 * q]);
+                hs[4 * q] = sc.x; hs[4 * q + 1] = sc.y; hs[4 * q + 2] = sc.z; hs[4 * q + 3] = sc.w;
+                hb[4 * q] = bi.x; hb[4 * q + 1] = bi.y; hb[4 * q + 2] = bi.z; hb[4 * q + 3] = bi.w;
+            }
         }
-        if (e.small_acc) {
-            v[4 * q + 0] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 0], sc.x, bi.x, relu_first));
-            v[4 * q + 1] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 1], sc.y, bi.y, relu_first));
-            v[4 * q + 2] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 2], sc.z, bi.z, relu_first));
-            v[4 * q + 3] = __float_as_uint(dequant<true>((int32_t)v[4 * q + 3], sc.w, bi.w, relu_first));
-        } else {
-            v[4 * q + 0] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 0], sc.x, bi.x, relu_first));
-            v[4 * q + 1] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 1], sc.y, bi.y, relu_first));
-            v[4 * q + 2] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 2], sc.z, bi.z, relu_first));
-            v[4 * q + 3] = __float_as_uint(dequant<false>((int32_t)v[4 * q + 3], sc.w, bi.w, relu_first));
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int c = 16 * h + i;
+            v[c] = __float_as_uint(e.small_acc ? dequant<true>((int32_t)v[c], hs[i], hb[i], relu_first)
+                                               : dequant<false>((int32_t)v[c], hs[i], hb[i], relu_first));
         }
     }
     if (e.residual) {
@@ -483,6 +489,32 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[NV], i
             for (int i = 0; i < NV && col0 + i < e.N; ++i)
                 e.u8_out[off + i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
         }
+    }
+}
+
+// A warp's share of one accumulator: CHUNKS chunks of 32 columns starting at tensor-memory
+// address taddr0 (tile-local column cbase), for this thread's output row.  After the last
+// chunk has landed in registers the warp hands the accumulator back by arriving on
+// acc_empty_bar.
+template <int CHUNKS>
+__device__ __forceinline__ void epi_warp_columns(const EpiView &e, uint32_t taddr0, int cbase, int64_t row, bool row_ok,
+                                                 int64_t n0, const float *s_scale, const float *s_bias,
+                                                 uint32_t acc_empty_bar, int lane)
+{
+#pragma unroll 1
+    for (int ch = 0; ch < CHUNKS; ++ch) {
+        uint32_t v[32];
+        tmem_ld_32x32_issue(taddr0 + (uint32_t)(ch * 32), v);
+        tmem_ld_wait();
+        if (ch + 1 == CHUNKS) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar);
+        }
+        const int ct = cbase + ch * 32;              // column inside the tile
+        const int64_t col0 = n0 + ct;
+        if (!row_ok || col0 >= e.N) continue;
+        epi_chunk<32, false>(e, v, row, col0, ct, s_scale, s_bias);
     }
 }
 
@@ -619,7 +651,10 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         __syncwarp();
     } else if (warp == 1) {
         // ================= MMA issuer =================
-        if (lane == 0) {
+        // The whole warp runs this loop converged and one elected lane issues, so that the
+        // descriptor arithmetic (warp-uniform values only) can stay in the uniform datapath.
+        {
+            const uint32_t elected = elect_one();
             constexpr uint32_t idesc = make_idesc_i8(BN);
             // descriptors of stage 0; a stage adds its byte offset / 16 to the start-address field
             const uint64_t adesc0 = make_smem_desc<BK>(smem_base);
@@ -643,18 +678,18 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     const uint64_t adesc = adesc0 + st_off, bdesc = bdesc0 + st_off;
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)
-                        tc_mma_i8(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
-                                  (kb > 0 || k > 0) ? 1u : 0u);
-                    tc_commit(smem_u32(&bar_empty[s]));       // stage reusable once these MMAs retire
+                        tc_mma_i8_if(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
+                                     (kb > 0 || k > 0) ? 1u : 0u, elected);
+                    tc_commit_if(smem_u32(&bar_empty[s]), elected);       // stage reusable once these MMAs retire
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
-                tc_commit(smem_u32(&bar_acc_full[acc]));      // accumulator complete
+                tc_commit_if(smem_u32(&bar_acc_full[acc]), elected);      // accumulator complete
             }
             SPARQ_PROF_STORE(2, mw);
             SPARQ_PROF_STORE(3, ma);
             SPARQ_PROF_STORE(4, SPARQ_PROF_NOW() - mt0);
             // all tensor-core work of this CTA has retired before tensor memory is freed
-            tc_commit(smem_u32(&bar_done));
+            tc_commit_if(smem_u32(&bar_done), elected);
             mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, true);
         }
         __syncwarp();
@@ -683,22 +718,8 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const bool row_ok = row < g.M;
             const int cbase = half * (BN / 2);
             const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + cbase);
-#pragma unroll 1
-            for (int ch = 0; ch < kChunks; ++ch) {
-                uint32_t v[32];
-                tmem_ld_32x32_issue(taddr0 + (uint32_t)(ch * 32), v);
-                tmem_ld_wait();
-                if (ch + 1 == kChunks) {
-                    // this warp's share of the accumulator is in registers: hand it back
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
-                }
-                const int ct = cbase + ch * 32;              // column inside the tile
-                const int64_t col0 = nt * BN + ct;
-                if (!row_ok || col0 >= g.N) continue;
-                epi_chunk(ev, v, row, col0, ct, s_scale, s_bias);
-            }
+            epi_warp_columns<kChunks>(ev, taddr0, cbase, row, row_ok, nt * BN, s_scale, s_bias,
+                                      smem_u32(&bar_acc_empty[acc]), lane);
         }
         if (warp == kFirstEpiWarp && lane == 0) {
             SPARQ_PROF_STORE(5, ew);
