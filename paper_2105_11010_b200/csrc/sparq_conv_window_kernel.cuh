@@ -114,7 +114,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&bar_acc_full[a]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[a]), kNumEpiWarps);
+            mbar_init(smem_u32(&bar_acc_empty[a]), epi_warps(MODE));
         }
         mbar_init(smem_u32(&bar_done), 1);
         abort_word = 0;
@@ -291,14 +291,15 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, true);
         }
         __syncwarp();
-    } else if (warp < kFirstXfWarp) {
+    } else if (warp < kFirstEpiWarp + epi_warps(MODE)) {
         // ================= epilogue =================
+        constexpr int kEpi = epi_warps(MODE);
+        constexpr int kColsPerWarp = BN / (kEpi / 4);     // the tile's columns are split over the warps of a quarter
         const int quarter = warp & 3;
-        const int half = (warp - kFirstEpiWarp) >> 2;
+        const int part = (warp - kFirstEpiWarp) >> 2;
         const int et = threadIdx.x - kFirstEpiWarp * 32;
         const EpiView ev = make_epi_view(g);
         uint32_t wt = 0;
-        constexpr int kChunks = BN / 64;
         int64_t staged_nt = -1;
         // this thread's slot inside a tile: row tr of the tile, padded column ow
         const int slot = quarter * 32 + lane;
@@ -307,17 +308,17 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         const bool slot_ok = (tr < g.TR) && (ow < g.Wo);
         long long ew = 0;
         const long long et0 = SPARQ_PROF_NOW();
-        // 64-wide tiles have one column tile and one 32-column chunk per warp.  When only the
+        // 64-wide tiles have one column tile and 16 or 32 columns per warp.  When only the
         // requantized bytes are wanted (the form every layer of a network uses), the warp keeps
-        // the scale and bias of its 32 columns in registers for the whole launch -- shared-memory
+        // the scale and bias of its columns in registers for the whole launch -- shared-memory
         // reads queue behind the tensor core's operand fetches -- and takes the accumulator in
-        // two 16-column halves so that those 64 registers fit beside it.
+        // 16-column pieces so that those registers fit beside it.
         if (BN == 64 && ev.need_f && !g.acc_out && !g.f32_out && !g.residual && g.N == 64) {
-            epi_stage_scale_bias(g, 0, BN, et, s_scale, s_bias);
-            const int cbase = half * 32;
-            float rs[32], rb[32];
+            epi_stage_scale_bias<kEpi>(g, 0, BN, et, s_scale, s_bias);
+            const int cbase = part * kColsPerWarp;
+            float rs[kColsPerWarp], rb[kColsPerWarp];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
+            for (int i = 0; i < kColsPerWarp; ++i) {
                 rs[i] = s_scale[cbase + i];
                 rb[i] = s_bias[cbase + i];
             }
@@ -333,11 +334,11 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt >> 1) & 1u, abort_flag, g.status));
                 tc_fence_after();
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
+                for (int hh = 0; hh < kColsPerWarp / 16; ++hh) {
                     uint32_t v[16];
                     tmem_ld_32x16_issue(taddr0 + (uint32_t)(hh * 16), v);
                     tmem_ld_wait();
-                    if (hh == 1) {
+                    if (hh + 1 == kColsPerWarp / 16) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
@@ -383,7 +384,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             const uint32_t acc_use = wt >> 1;
             if (ev.need_f && nt != staged_nt) {
                 staged_nt = nt;
-                epi_stage_scale_bias(g, nt * BN, BN, et, s_scale, s_bias);
+                epi_stage_scale_bias<kEpi>(g, nt * BN, BN, et, s_scale, s_bias);
             }
             SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status));
             tc_fence_after();
@@ -391,9 +392,9 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             const int oh = (int)(mt % g.tiles_per_img) * g.TR + tr;
             const bool row_ok = slot_ok && (oh < g.Ho);
             const int64_t row = ((int64_t)img * g.Ho + oh) * g.Wo + ow;
-            const int cbase = half * (BN / 2);
+            const int cbase = part * kColsPerWarp;
             const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + cbase);
-            epi_warp_columns<kChunks>(ev, taddr0, cbase, row, row_ok, nt * BN, s_scale, s_bias,
+            epi_warp_columns<kColsPerWarp>(ev, taddr0, cbase, row, row_ok, nt * BN, s_scale, s_bias,
                                       smem_u32(&bar_acc_empty[acc]), lane);
         }
         if (warp == kFirstEpiWarp && lane == 0) {

@@ -31,11 +31,14 @@
 namespace sparq {
 
 constexpr int kBM = 128;                 // rows of an output tile = MMA M
-constexpr int kNumEpiWarps = 8;          // two per tensor-memory lane quarter
+constexpr int kNumEpiWarps = 8;          // two per tensor-memory lane quarter; without a transform
+                                         // (mode NONE) the transform warps are epilogue warps too
 constexpr int kNumXfWarps = 8;
 constexpr int kFirstEpiWarp = 2;
 constexpr int kFirstXfWarp = kFirstEpiWarp + kNumEpiWarps;
 constexpr int kGemmThreads = 32 * (kFirstXfWarp + kNumXfWarps);
+// Epilogue warps of a kernel instantiated for `mode`.
+__host__ __device__ constexpr int epi_warps(int mode) { return mode == SPARQ_MODE_NONE ? kNumEpiWarps + kNumXfWarps : kNumEpiWarps; }
 constexpr int kSmemBudget = 200 * 1024;  // for the stage ring
 constexpr long long kWaitLimitCycles = 2000000000LL;
 
@@ -247,9 +250,10 @@ __device__ __forceinline__ constexpr uint32_t make_idesc_i8(int n)
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Barrier among the epilogue warps only (hardware barrier 1).
+template <int WARPS>
 __device__ __forceinline__ void epi_bar_sync()
 {
-    asm volatile("bar.sync 1, %0;" :: "n"(kNumEpiWarps * 32) : "memory");
+    asm volatile("bar.sync 1, %0;" :: "n"(WARPS * 32) : "memory");
 }
 
 // 32 contiguous bytes with one 256-bit store (dst 32-byte aligned).
@@ -492,45 +496,57 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[NV], i
     }
 }
 
-// A warp's share of one accumulator: CHUNKS chunks of 32 columns starting at tensor-memory
-// address taddr0 (tile-local column cbase), for this thread's output row.  After the last
-// chunk has landed in registers the warp hands the accumulator back by arriving on
-// acc_empty_bar.
-template <int CHUNKS>
+// A warp's share of one accumulator: CW (16, 32, 64 or 128) columns starting at
+// tensor-memory address taddr0 (tile-local column cbase), for this thread's output row.
+// After the last load has landed in registers the warp hands the accumulator back by
+// arriving on acc_empty_bar.
+template <int CW>
 __device__ __forceinline__ void epi_warp_columns(const EpiView &e, uint32_t taddr0, int cbase, int64_t row, bool row_ok,
                                                  int64_t n0, const float *s_scale, const float *s_bias,
                                                  uint32_t acc_empty_bar, int lane)
 {
-#pragma unroll 1
-    for (int ch = 0; ch < CHUNKS; ++ch) {
-        uint32_t v[32];
-        tmem_ld_32x32_issue(taddr0 + (uint32_t)(ch * 32), v);
+    if constexpr (CW == 16) {
+        uint32_t v[16];
+        tmem_ld_32x16_issue(taddr0, v);
         tmem_ld_wait();
-        if (ch + 1 == CHUNKS) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty_bar);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty_bar);
+        const int64_t col0 = n0 + cbase;
+        if (row_ok && col0 < e.N) epi_chunk<16, false>(e, v, row, col0, cbase, s_scale, s_bias);
+    } else {
+        constexpr int CHUNKS = CW / 32;
+#pragma unroll 1
+        for (int ch = 0; ch < CHUNKS; ++ch) {
+            uint32_t v[32];
+            tmem_ld_32x32_issue(taddr0 + (uint32_t)(ch * 32), v);
+            tmem_ld_wait();
+            if (ch + 1 == CHUNKS) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty_bar);
+            }
+            const int ct = cbase + ch * 32;              // column inside the tile
+            const int64_t col0 = n0 + ct;
+            if (!row_ok || col0 >= e.N) continue;
+            epi_chunk<32, false>(e, v, row, col0, ct, s_scale, s_bias);
         }
-        const int ct = cbase + ch * 32;              // column inside the tile
-        const int64_t col0 = n0 + ct;
-        if (!row_ok || col0 >= e.N) continue;
-        epi_chunk<32, false>(e, v, row, col0, ct, s_scale, s_bias);
     }
 }
 
 // Stages the scale and bias of columns n0 .. n0+bn-1 in shared memory (epilogue warps only).
-template <class Args>
+template <int WARPS, class Args>
 __device__ __forceinline__ void epi_stage_scale_bias(const Args &g, int64_t n0, int bn, int et,
                                                      float *s_scale, float *s_bias)
 {
-    epi_bar_sync();                             // previous readers are done
-    for (int c = et; c < bn; c += kNumEpiWarps * 32) {
+    epi_bar_sync<WARPS>();                      // previous readers are done
+    for (int c = et; c < bn; c += WARPS * 32) {
         const int64_t col = n0 + c;
         const bool ok = col < g.N;
         s_scale[c] = ok ? __ldg(g.scale + col) : 0.0f;
         s_bias[c] = (ok && g.bias) ? __ldg(g.bias + col) : 0.0f;
     }
-    epi_bar_sync();
+    epi_bar_sync<WARPS>();
 }
 
 // ---- the kernel ---------------------------------------------------------------------------
@@ -579,7 +595,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&bar_acc_full[a]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[a]), kNumEpiWarps);
+            mbar_init(smem_u32(&bar_acc_empty[a]), epi_warps(MODE));
         }
         mbar_init(smem_u32(&bar_done), 1);
         abort_word = 0;
@@ -693,14 +709,15 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, true);
         }
         __syncwarp();
-    } else if (warp < kFirstXfWarp) {
+    } else if (warp < kFirstEpiWarp + epi_warps(MODE)) {
         // ================= epilogue =================
+        constexpr int kEpi = epi_warps(MODE);
+        constexpr int kColsPerWarp = BN / (kEpi / 4);        // the tile's columns are split over the warps of a quarter
         const int quarter = warp & 3;                        // tensor-memory lanes this warp may read
-        const int half = (warp - kFirstEpiWarp) >> 2;        // which half of the tile's columns
-        const int et = threadIdx.x - kFirstEpiWarp * 32;     // 0 .. 255
+        const int part = (warp - kFirstEpiWarp) >> 2;        // which share of the tile's columns
+        const int et = threadIdx.x - kFirstEpiWarp * 32;     // 0 .. kEpi * 32 - 1
         const EpiView ev = make_epi_view(g);
         uint32_t local_tile = 0;
-        constexpr int kChunks = BN / 64;                     // 32-column chunks per warp
         int64_t staged_nt = -1;
         long long ew = 0;
         const long long et0 = SPARQ_PROF_NOW();
@@ -710,15 +727,15 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const uint32_t acc_use = local_tile >> 1;
             if (ev.need_f && nt != staged_nt) {              // new column tile: new scale / bias
                 staged_nt = nt;
-                epi_stage_scale_bias(g, nt * BN, BN, et, s_scale, s_bias);
+                epi_stage_scale_bias<kEpi>(g, nt * BN, BN, et, s_scale, s_bias);
             }
             SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status));
             tc_fence_after();
             const int64_t row = mt * kBM + quarter * 32 + lane;
             const bool row_ok = row < g.M;
-            const int cbase = half * (BN / 2);
+            const int cbase = part * kColsPerWarp;
             const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + cbase);
-            epi_warp_columns<kChunks>(ev, taddr0, cbase, row, row_ok, nt * BN, s_scale, s_bias,
+            epi_warp_columns<kColsPerWarp>(ev, taddr0, cbase, row, row_ok, nt * BN, s_scale, s_bias,
                                       smem_u32(&bar_acc_empty[acc]), lane);
         }
         if (warp == kFirstEpiWarp && lane == 0) {
