@@ -59,7 +59,6 @@ struct WindowArgs {
 constexpr int kWindowMaxDynSmem = 232448 - 4096;
 constexpr int kMaxWinBufs = 4;
 constexpr int kMaxBStages = 8;
-constexpr int kMaxKb = 128;     // (tap, channel block) pairs the MMA warp keeps a table for
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w, int h, int n)
 {
@@ -80,9 +79,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
     __shared__ uint32_t tmem_base_slot;
     __shared__ uint32_t abort_word;
     __shared__ __align__(16) float s_scale[BN], s_bias[BN];
-    // per (channel block, tap): .x = offset of the tap's A rows inside a window buffer,
-    // .y = offset of the resident weight block; both in 16-byte units (descriptor units)
-    __shared__ uint2 s_tab[kMaxKb];
 
     constexpr int kBBlock = BN * CB;                   // one (tap, channel block) of weights
     constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;
@@ -121,12 +117,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        for (int kb = lane; kb < kb_count; kb += 32) {
-            const int cb = kb / taps, tap = kb % taps;
-            const uint32_t rows = (uint32_t)((tap / g.S) * g.Wp + (tap % g.S));
-            s_tab[kb] = make_uint2(((uint32_t)cb * (uint32_t)g.plane_bytes + rows * CB) >> 4,
-                                   (uint32_t)kb * (uint32_t)(kBBlock >> 4));
-        }
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      :: "r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -226,17 +216,9 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             int s = 0;  uint32_t bph = 0;      // streamed weight stage and its phase parity
             long long mw = 0, ma = 0, mb = 0, mi = 0;
             const long long mt0 = SPARQ_PROF_NOW();
-            constexpr int kRegTab = 18;         // 3x3 taps of up to two channel blocks
-            uint2 rtab[kRegTab];
-#pragma unroll
-            for (int kb = 0; kb < kRegTab; ++kb) {
-                // same entries as s_tab, from the kernel arguments
-                const int cb = kb / taps, tap = kb % taps;
-                const uint32_t rows = (uint32_t)((tap / g.S) * g.Wp + (tap % g.S));
-                rtab[kb] = (kb < kb_count) ? make_uint2(((uint32_t)cb * (uint32_t)g.plane_bytes + rows * CB) >> 4,
-                                                        (uint32_t)kb * (uint32_t)(kBBlock >> 4))
-                                           : make_uint2(0u, 0u);
-            }
+            // descriptor steps, in 16-byte units: one padded input row, one channel-block plane
+            const uint32_t row16 = (uint32_t)(g.Wp * CB) >> 4;
+            const uint32_t plane16 = (uint32_t)g.plane_bytes >> 4;
             if (B_RESIDENT) SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status));
             for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
                 const int acc = wt & 1;
@@ -249,17 +231,18 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 const uint64_t a_desc0 = win_desc0 + (uint64_t)((uint32_t)b * (win_bytes >> 4));
                 const long long is0 = SPARQ_PROF_NOW();
                 // One (tap, channel block) of the tile: wait for its weights when they are
-                // streamed, then CB / 32 MMAs.
-                auto issue_block = [&](int kb, const uint2 e) {
+                // streamed, then CB / 32 MMAs.  The descriptors are sums of warp-uniform
+                // loop-carried values (no table, no division), so the address arithmetic of
+                // consecutive MMAs is a couple of adds.
+                auto issue_block = [&](const uint32_t kb, const uint64_t adesc) {
                     uint64_t bdesc;
                     if (B_RESIDENT) {
-                        bdesc = b_desc0 + (uint64_t)e.y;
+                        bdesc = b_desc0 + (uint64_t)(kb * (uint32_t)(kBBlock >> 4));
                     } else {
                         SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status));
                         tc_fence_after();
                         bdesc = b_desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kBBlock >> 4));
                     }
-                    const uint64_t adesc = a_desc0 + (uint64_t)e.x;
 #pragma unroll
                     for (int k = 0; k < CB / 32; ++k)
                         tc_mma_i8_if(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
@@ -269,13 +252,23 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                         if (++s == g.b_stages) { s = 0; bph ^= 1u; }
                     }
                 };
-                if (kb_count <= kRegTab) {
-                    // table in registers: nothing but two adds stands between consecutive MMAs
+                uint32_t kb = 0;
+                uint64_t a_cb = a_desc0;
+                if (g.R == 3 && g.S == 3) {
+                    for (int cb = 0; cb < g.c_blocks; ++cb, a_cb += plane16) {
 #pragma unroll
-                    for (int kb = 0; kb < kRegTab; ++kb)
-                        if (kb < kb_count) issue_block(kb, rtab[kb]);
+                        for (int r = 0; r < 3; ++r)
+#pragma unroll
+                            for (int sx = 0; sx < 3; ++sx, ++kb)
+                                issue_block(kb, a_cb + (uint64_t)((uint32_t)r * row16 + (uint32_t)(sx * (CB >> 4))));
+                    }
                 } else {
-                    for (int kb = 0; kb < kb_count; ++kb) issue_block(kb, s_tab[kb]);
+                    for (int cb = 0; cb < g.c_blocks; ++cb, a_cb += plane16) {
+                        uint64_t a_r = a_cb;
+                        for (int r = 0; r < g.R; ++r, a_r += row16)
+                            for (int sx = 0; sx < g.S; ++sx, ++kb)
+                                issue_block(kb, a_r + (uint64_t)(uint32_t)(sx * (CB >> 4)));
+                    }
                 }
                 mi += SPARQ_PROF_NOW() - is0;
                 tc_commit_if(smem_u32(&bar_win_empty[b]), elected);       // window reusable once these MMAs retire

@@ -257,7 +257,6 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     const int c_blocks = c / cb;
     const int taps = r * s;
     const int kb_count = taps * c_blocks;
-    if (kb_count > kMaxKb) return 0;
     const int rows_alloc = (r - 1) * wp + (s - 1) + 128;
     // a plane holds every row the MMA may touch and the whole 16 KB groups the transform rewrites
     const int box_bytes = cb * wp * (tr + r - 1);
