@@ -1,19 +1,28 @@
-// Stride-1 R x S convolution with the activation transform applied ONCE per staged input
-// pixel ("window" kernel).
+// Stride-1 R x S convolution with the activation transform applied once per staged input
+// row ("window" kernel).
 //
 // The im2col form of the fused kernel stages a shifted copy of the input for every filter
 // tap, so every input byte is copied into shared memory and transformed R*S times.  Here a
 // CTA's output tile is TR whole output rows of one image, laid out with the PADDED width
 // Wp = W + 2*pad_w (slot i = tr * Wp + ow; the S-1 slots at the end of each row are junk and
 // are never stored).  With that layout tap (r, s) of slot i reads padded-input pixel
-// i + r*Wp + s: every tap is the SAME shared-memory matrix shifted by r*Wp + s rows.  So
-//   * one tiled TMA box (CB channels x Wp x (TR+R-1) rows, zero fill outside the image)
-//     brings the tile's input window in once per channel block,
-//   * the transform warps rewrite it in place once (bSPARQ / vSPARQ, Sections 3.1-3.2),
+// i + r*Wp + s: every tap is the SAME shared-memory matrix shifted by r*Wp + s rows.
+//
+// Up to G consecutive tiles of one image form a GROUP that shares one window buffer of
+// G*TR + R-1 input rows, so the R-1 halo rows between neighbouring tiles are staged and
+// transformed once instead of once per tile.  The window arrives in pieces -- the first is
+// TR+R-1 rows, every later one TR rows -- each with its own pair of barriers, and tile j of
+// the group needs pieces 0..j only: the tensor core starts on the first tile while later
+// pieces are still in flight or being transformed.
+//   * tiled TMA boxes (CB channels x Wp x piece rows, zero fill outside the image) bring the
+//     pieces in, once per channel block; the swizzle of a box is a function of the
+//     shared-memory address, so pieces written at consecutive row offsets form one
+//     consistently swizzled matrix,
+//   * the transform warps rewrite each piece in place once (bSPARQ / vSPARQ, Sections 3.1-3.2),
 //   * the MMA warp issues tcgen05.mma kind::i8 for every (channel block, tap) with an A
-//     descriptor whose start address is advanced by (r*Wp + s) rows.  The 128-/64-byte
-//     swizzle is a function of the shared-memory address, so a row-shifted start reads the
-//     bytes TMA wrote.
+//     descriptor whose start address is advanced by (j*TR*Wp + r*Wp + s) rows.
+// Each CTA owns a contiguous range of the tile sequence (balanced to within one tile) and
+// cuts it into groups at image boundaries.
 // Weights either stay resident in shared memory for the whole kernel (B_RESIDENT: all
 // R*S*C/CB blocks of BN x CB, loaded once per CTA) or stream through a ring of stages.
 // Warp roles, bounded waits and the epilogue are those of sparq_gemm_kernel.
@@ -33,10 +42,16 @@ struct WindowArgs {
     int TR;                 // output rows per tile
     int tiles_per_img;      // ceil(Ho / TR)
     int c_blocks;           // C / CB
-    int box_bytes;          // CB * Wp * (TR + R - 1): one channel block of one tile's window
+    int G;                  // most tiles that share one window (1 when there are several column tiles)
+    int piece0_bytes;       // CB * Wp * (TR + R - 1): first piece of a group, one channel block
+    int piece_bytes;        // CB * Wp * TR: every later piece
     int plane_bytes;        // shared-memory bytes reserved per channel block (>= rows the MMA may touch)
     int win_bufs;           // window buffers in the ring
     int b_stages;           // weight stages (stream mode) or resident blocks (resident mode)
+    int issuers;            // 1: warp 1 issues every tile; 2: the two issuer warps alternate
+    int w_one_copy;         // resident weights: map_w is the 3-D (bytes, rows, blocks) view and one copy brings all blocks
+    uint32_t n_tiles;       // column tiles
+    uint32_t units;         // n_img * tiles_per_img * n_tiles, column tile fastest
     // transform
     XformDev xf;
     // epilogue
@@ -58,7 +73,14 @@ struct WindowArgs {
 // dynamic shared memory the kernel may ask for: 227 KB minus room for its static variables
 constexpr int kWindowMaxDynSmem = 232448 - 4096;
 constexpr int kMaxWinBufs = 4;
+constexpr int kMaxG = 8;
 constexpr int kMaxBStages = 8;
+// Two warps issue MMAs, taking the tiles of a CTA alternately (each owns one of the two
+// accumulators): whatever one of them does between two tiles -- commits, barrier reads that
+// queue behind the tensor core's own shared-memory traffic, descriptor set-up -- happens
+// while the other one's MMAs keep the tensor core busy.
+constexpr int kMmaBWarp = kFirstXfWarp + kNumXfWarps;      // the second issuer is the last warp
+constexpr int kWindowThreads = kGemmThreads + 32;
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w, int h, int n)
 {
@@ -67,21 +89,70 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
         :: "r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
+// Walks the groups of one CTA's share of the tile sequence.  Every warp role runs the same
+// walk, so that window buffers, accumulators and barrier phases line up without any
+// communication.
+struct GroupWalk {
+    uint32_t u, u_end;          // units still to do: [u, u_end)
+    uint32_t n_tiles, tpi, G;
+    uint32_t img, tin, nt, cnt; // current group: image, first tile inside it, column tile, tiles
+
+    __device__ __forceinline__ GroupWalk(const WindowArgs &g)
+    {
+        // units split into gridDim.x contiguous shares that differ by at most one
+        const uint32_t q = g.units / gridDim.x, rem = g.units - q * gridDim.x;
+        u = blockIdx.x * q + (blockIdx.x < rem ? blockIdx.x : rem);
+        u_end = u + q + (blockIdx.x < rem ? 1u : 0u);
+        n_tiles = g.n_tiles; tpi = (uint32_t)g.tiles_per_img; G = (uint32_t)g.G;
+        img = tin = nt = cnt = 0;
+    }
+    __device__ __forceinline__ bool next()
+    {
+        if (u >= u_end) return false;
+        uint32_t mt = u;
+        nt = 0;
+        if (n_tiles != 1) { mt = u / n_tiles; nt = u - mt * n_tiles; }
+        img = mt / tpi;
+        tin = mt - img * tpi;
+        uint32_t c = 1;
+        if (n_tiles == 1) {
+            c = tpi - tin;
+            if (c > G) c = G;
+            if (c > u_end - u) c = u_end - u;
+        }
+        cnt = c;
+        u += c;
+        return true;
+    }
+};
+
 template <int BN, int CB, int MODE, int XN, bool RND, bool B_RESIDENT>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                         const WindowArgs g)
+__global__ void __launch_bounds__(kWindowThreads, 1)
+sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __grid_constant__ CUtensorMap map_x1,
+                         const __grid_constant__ CUtensorMap map_w, const WindowArgs g)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_win_full[kMaxWinBufs], bar_win_xf[kMaxWinBufs], bar_win_empty[kMaxWinBufs];
+    // one pair per (window buffer, piece): bytes landed / piece transformed
+    __shared__ __align__(8) uint64_t bar_win_full[kMaxWinBufs * kMaxG], bar_win_xf[kMaxWinBufs * kMaxG];
+    __shared__ __align__(8) uint64_t bar_win_empty[kMaxWinBufs];
     __shared__ __align__(8) uint64_t bar_b_full[kMaxBStages], bar_b_empty[kMaxBStages];
-    __shared__ __align__(8) uint64_t bar_acc_full[2], bar_acc_empty[2], bar_done;
+    // Accumulator stages in tensor memory; tile number t uses stage t % kAcc.  (Four stages were
+    // measured and changed nothing: the epilogue hands a stage back well within one tile.)
+    constexpr int kAcc = 2;
+    __shared__ __align__(8) uint64_t bar_acc_full[kAcc], bar_acc_empty[kAcc], bar_done;
     __shared__ uint32_t tmem_base_slot;
     __shared__ uint32_t abort_word;
     __shared__ __align__(16) float s_scale[BN], s_bias[BN];
 
     constexpr int kBBlock = BN * CB;                   // one (tap, channel block) of weights
-    constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;
+    constexpr int kTmemCols = kAcc * BN;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     volatile uint32_t *abort_flag = &abort_word;
@@ -92,28 +163,37 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
     auto win_buf = [&](int b) { return smem_base + (uint32_t)b * win_bytes; };
     const uint32_t b_base = smem_base + (uint32_t)g.win_bufs * win_bytes;
     auto b_slot = [&](int s) { return b_base + (uint32_t)s * kBBlock; };
+    // byte offset of piece j inside a channel block's plane, and its size
+    auto piece_off = [&](int j) { return j ? (uint32_t)((j * g.TR + g.R - 1) * g.Wp * CB) : 0u; };
+    auto piece_len = [&](int j) { return (uint32_t)(j ? g.piece_bytes : g.piece0_bytes); };
 
     const int taps = g.R * g.S;
     const int kb_count = taps * g.c_blocks;            // weight blocks per tile
 
     if (threadIdx.x == 0) {
-        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_x0);
+        prefetch_tensormap(&map_x1);
         prefetch_tensormap(&map_w);
-        for (int b = 0; b < kMaxWinBufs; ++b) {
+    }
+    if (warp == 0) {
+        // barrier set-up spread over the lanes of one warp
+        for (int b = lane; b < kMaxWinBufs * kMaxG; b += 32) {
             mbar_init(smem_u32(&bar_win_full[b]), 1);
             mbar_init(smem_u32(&bar_win_xf[b]), kNumXfWarps);
-            mbar_init(smem_u32(&bar_win_empty[b]), 1);
         }
-        for (int s = 0; s < kMaxBStages; ++s) {
-            mbar_init(smem_u32(&bar_b_full[s]), 1);
-            mbar_init(smem_u32(&bar_b_empty[s]), 1);
+        if (lane < kMaxWinBufs) mbar_init(smem_u32(&bar_win_empty[lane]), 2);     // one arrival per issuing warp
+        if (lane < kMaxBStages) {
+            mbar_init(smem_u32(&bar_b_full[lane]), 1);
+            mbar_init(smem_u32(&bar_b_empty[lane]), 1);
         }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(smem_u32(&bar_acc_full[a]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[a]), epi_warps(MODE));
+        if (lane < kAcc) {
+            mbar_init(smem_u32(&bar_acc_full[lane]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[lane]), epi_warps(MODE));
         }
-        mbar_init(smem_u32(&bar_done), 1);
-        abort_word = 0;
+        if (lane == 0) {
+            mbar_init(smem_u32(&bar_done), 2);
+            abort_word = 0;
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -128,160 +208,262 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
     dep_launch();
     dep_wait();
 
-    // With resident weights there is one column tile (host guarantees N <= BN).
-    const int64_t n_tiles = (g.N + BN - 1) / BN;
-    const int64_t m_tiles = (int64_t)g.n_img * g.tiles_per_img;
-    const int64_t total_tiles = m_tiles * n_tiles;
+    GroupWalk walk(g);
+    if (threadIdx.x == 0) SPARQ_PROF_STORE(15, SPARQ_PROF_NOW() - cta_t0);
 
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            uint32_t wt = 0;      // window counter
+            uint32_t gi = 0;      // group counter
             uint32_t it = 0;      // streamed weight-block counter
             bool b_issued = false;  // resident weights requested
             long long pw = 0;
             const long long pt0 = SPARQ_PROF_NOW();
-            for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
-                const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
-                const int img = (int)(mt / g.tiles_per_img);
-                const int oh0 = (int)(mt % g.tiles_per_img) * g.TR;
-                const int b = wt % g.win_bufs;
-                const uint32_t use = wt / g.win_bufs;
+            while (walk.next()) {
+                const int b = gi % g.win_bufs;
+                const uint32_t use = gi / g.win_bufs;
                 if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_win_empty[b]), (use - 1) & 1, abort_flag, g.status));
                 if (*abort_flag) break;
-                const uint32_t wfull = smem_u32(&bar_win_full[b]);
-                mbar_expect_tx(wfull, (uint32_t)g.box_bytes * (uint32_t)g.c_blocks);
-                for (int cb = 0; cb < g.c_blocks; ++cb)
-                    tma_load_4d(win_buf(b) + (uint32_t)cb * g.plane_bytes, &map_x, wfull,
-                                cb * CB, -g.pad_w, oh0 - g.pad_h, img);
-                if (B_RESIDENT && wt == 0) {
-                    // all weight blocks, once per CTA, on stage barrier 0 -- after the first
-                    // window so that the activations (which come from HBM and still have to
-                    // be transformed) are requested first
+                const int oh0 = (int)walk.tin * g.TR;
+                if (gi == 0) SPARQ_PROF_STORE(9, SPARQ_PROF_NOW() - pt0);
+                if (B_RESIDENT && !b_issued) {
+                    // All weight blocks, once per CTA, on stage barrier 0, ahead of the first
+                    // window: every CTA reads the same bytes, so they come out of L2 one reader
+                    // after the other and are the last thing the first tile waits for.  Block
+                    // (tap, cb) = bytes [tap*C + cb*CB, +CB) of every filter lands in slot
+                    // tap * c_blocks + cb.
                     const uint32_t full = smem_u32(&bar_b_full[0]);
                     mbar_expect_tx(full, (uint32_t)kb_count * kBBlock);
-                    for (int kb = 0; kb < kb_count; ++kb) {
-                        const int cb = kb / taps, tap = kb % taps;
-                        tma_load_2d(b_slot(kb), &map_w, full, tap * g.C + cb * CB, 0);
+                    if (g.w_one_copy) {
+                        tma_load_3d(b_slot(0), &map_w, full, 0, 0, 0);
+                    } else {
+                        for (int kb = 0; kb < kb_count; ++kb) tma_load_2d(b_slot(kb), &map_w, full, kb * CB, 0);
                     }
                     b_issued = true;
+                    SPARQ_PROF_STORE(14, SPARQ_PROF_NOW() - pt0);
                 }
-                if (!B_RESIDENT) {
-                    for (int kb = 0; kb < kb_count; ++kb, ++it) {
-                        const int s = it % g.b_stages;
-                        const uint32_t buse = it / g.b_stages;
-                        if (buse > 0) mbar_wait(smem_u32(&bar_b_empty[s]), (buse - 1) & 1, abort_flag, g.status);
-                        if (*abort_flag) break;
-                        const int cb = kb / taps, tap = kb % taps;
-                        const uint32_t full = smem_u32(&bar_b_full[s]);
-                        mbar_expect_tx(full, kBBlock);
-                        tma_load_2d(b_slot(s), &map_w, full, tap * g.C + cb * CB, (int)(nt * BN));
+                for (int j = 0; j < g.G; ++j) {
+                    const uint32_t wfull = smem_u32(&bar_win_full[b * kMaxG + j]);
+                    if (j < (int)walk.cnt) {
+                        mbar_expect_tx(wfull, piece_len(j) * (uint32_t)g.c_blocks);
+                        const int h0 = oh0 - g.pad_h + (j ? j * g.TR + g.R - 1 : 0);
+                        uint32_t dst = win_buf(b) + piece_off(j);
+                        for (int cb = 0; cb < g.c_blocks; ++cb, dst += (uint32_t)g.plane_bytes)
+                            tma_load_4d(dst, j ? &map_x1 : &map_x0, wfull, cb * CB, -g.pad_w, h0, (int)walk.img);
+                    } else {
+                        // a piece this group does not have: complete its phase so that the
+                        // parity of every barrier of the buffer advances once per use
+                        mbar_arrive(wfull);
+                    }
+                    if (gi == 0 && j == 0) SPARQ_PROF_STORE(13, SPARQ_PROF_NOW() - pt0);
+                }
+#ifdef SPARQ_PROF
+                if (gi == 0) {
+                    SPARQ_PROF_TL(3, 1, cta_t0);
+                    for (int j = 0; j < (int)walk.cnt; ++j) {
+                        mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), 0, abort_flag, g.status);
+                        SPARQ_PROF_TL(3, 2 + j, cta_t0);
                     }
                 }
-                // an abort noticed here is acted on at the top of the next iteration, after this
-                // tile's window has been counted in wt (the drain below waits for it)
+#endif
+                ++gi;
+                if (!B_RESIDENT) {
+                    bool stop = false;
+                    for (int j = 0; j < (int)walk.cnt && !stop; ++j) {
+                        for (int cb = 0; cb < g.c_blocks && !stop; ++cb) {
+                            for (int tap = 0; tap < taps; ++tap, ++it) {
+                                const int s = it % g.b_stages;
+                                const uint32_t buse = it / g.b_stages;
+                                if (buse > 0) mbar_wait(smem_u32(&bar_b_empty[s]), (buse - 1) & 1, abort_flag, g.status);
+                                if (*abort_flag) { stop = true; break; }
+                                const uint32_t full = smem_u32(&bar_b_full[s]);
+                                mbar_expect_tx(full, kBBlock);
+                                tma_load_2d(b_slot(s), &map_w, full, tap * g.C + cb * CB, (int)(walk.nt * BN));
+                            }
+                        }
+                    }
+                    if (stop) break;
+                }
             }
             SPARQ_PROF_STORE(0, pw);
             SPARQ_PROF_STORE(1, SPARQ_PROF_NOW() - pt0);
             if (*abort_flag) {
                 // wait (bounded) for copies still in flight so that none lands after exit
-                const uint32_t wfirst = wt > (uint32_t)g.win_bufs ? wt - g.win_bufs : 0;
-                for (uint32_t j = wfirst; j < wt; ++j)
-                    mbar_wait(smem_u32(&bar_win_full[j % g.win_bufs]), (j / g.win_bufs) & 1, abort_flag, g.status, true);
+                const uint32_t gfirst = gi > (uint32_t)g.win_bufs ? gi - g.win_bufs : 0;
+                for (uint32_t q = gfirst; q < gi; ++q)
+                    for (int j = 0; j < g.G; ++j)
+                        mbar_wait(smem_u32(&bar_win_full[(q % g.win_bufs) * kMaxG + j]), (q / g.win_bufs) & 1,
+                                  abort_flag, g.status, true);
                 if (B_RESIDENT) {
-                    // the weight copies were issued together with the first window
                     if (b_issued) mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, true);
                 } else {
                     const uint32_t first = it > (uint32_t)g.b_stages ? it - g.b_stages : 0;
-                    for (uint32_t j = first; j < it; ++j)
-                        mbar_wait(smem_u32(&bar_b_full[j % g.b_stages]), (j / g.b_stages) & 1, abort_flag, g.status, true);
+                    for (uint32_t q = first; q < it; ++q)
+                        mbar_wait(smem_u32(&bar_b_full[q % g.b_stages]), (q / g.b_stages) & 1, abort_flag, g.status, true);
                 }
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // ================= MMA issuer =================
-        // The whole warp runs this loop converged and one elected lane issues: the descriptor
-        // arithmetic below is on warp-uniform values only (kernel arguments, loop counters),
-        // which lets it stay in the uniform datapath that feeds tcgen05.mma.
+    } else if (warp == 1 || warp == kMmaBWarp) {
+        // ================= MMA issuers =================
+        // Issuer `me` (0: warp 1, 1: the last warp) takes the tiles whose running number has
+        // parity `me`; tile number t goes into accumulator stage t % kAcc.  Each warp runs its loop converged and one elected
+        // lane issues: the descriptor arithmetic below is on warp-uniform values only (kernel
+        // arguments, loop counters), which lets it stay in the uniform datapath that feeds
+        // tcgen05.mma.
         {
+            const uint32_t me = (warp == 1) ? 0u : 1u;
             const uint32_t elected = elect_one();
             constexpr uint32_t idesc = make_idesc_i8(BN);
             // descriptors of window buffer 0 and of weight slot 0; offsets are added in units of
             // 16 bytes to the start-address field (the low word never carries into the next field)
             const uint64_t win_desc0 = make_smem_desc<CB>(smem_base);
             const uint64_t b_desc0 = make_smem_desc<CB>(b_base);
-            uint32_t wt = 0;
-            int b = 0;  uint32_t wph = 0;      // window buffer and its phase parity
+            uint32_t wt = 0;                   // tile counter (both issuers count every tile)
+            uint32_t gi = 0;                   // group counter (window buffer and phase)
             int s = 0;  uint32_t bph = 0;      // streamed weight stage and its phase parity
             long long mw = 0, ma = 0, mb = 0, mi = 0;
             const long long mt0 = SPARQ_PROF_NOW();
-            // descriptor steps, in 16-byte units: one padded input row, one channel-block plane
+            // descriptor steps, in 16-byte units: one padded input row, one channel-block plane,
+            // the rows of one tile
             const uint32_t row16 = (uint32_t)(g.Wp * CB) >> 4;
             const uint32_t plane16 = (uint32_t)g.plane_bytes >> 4;
+            const uint32_t tile16 = (uint32_t)(g.TR * g.Wp * CB) >> 4;
             if (B_RESIDENT) SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status));
-            for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
-                const int acc = wt & 1;
-                const uint32_t acc_use = wt >> 1;
-                if (acc_use > 0) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status));
-                if (MODE == SPARQ_MODE_NONE) SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_full[b]), wph, abort_flag, g.status));
-                else SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b]), wph, abort_flag, g.status));
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                const uint64_t a_desc0 = win_desc0 + (uint64_t)((uint32_t)b * (win_bytes >> 4));
-                const long long is0 = SPARQ_PROF_NOW();
-                // One (tap, channel block) of the tile: wait for its weights when they are
-                // streamed, then CB / 32 MMAs.  The descriptors are sums of warp-uniform
-                // loop-carried values (no table, no division), so the address arithmetic of
-                // consecutive MMAs is a couple of adds.
-                auto issue_block = [&](const uint32_t kb, const uint64_t adesc) {
-                    uint64_t bdesc;
-                    if (B_RESIDENT) {
-                        bdesc = b_desc0 + (uint64_t)(kb * (uint32_t)(kBBlock >> 4));
+            while (walk.next()) {
+                const int b = gi % g.win_bufs;
+                const uint32_t wph = (gi / g.win_bufs) & 1u;
+                const uint64_t a_grp = win_desc0 + (uint64_t)((uint32_t)b * (win_bytes >> 4));
+                bool issued = false;
+                // Barrier reads go through the shared-memory pipe, which the tensor core's operand
+                // fetches keep saturated, so a read takes hundreds of cycles.  The two barriers of
+                // this issuer's NEXT tile of the group are therefore looked at (non-blocking, both
+                // reads in flight together) after the first few MMAs of the current tile have been
+                // queued; when both say "ready" -- the usual case -- that tile starts without
+                // touching shared memory.
+                uint32_t pre_acc = 0, pre_ops = 0;
+                for (int j = 0; j < (int)walk.cnt; ++j, ++wt) {
+                    if (g.issuers == 2 ? (wt & 1u) != me : me != 0u) {
+                        if (!B_RESIDENT) {
+                            // the other issuer consumes this tile's weight stages
+                            s += kb_count;
+                            while (s >= g.b_stages) { s -= g.b_stages; bph ^= 1u; }
+                        }
+                        continue;
+                    }
+                    issued = true;
+                    const uint32_t acc = wt & (uint32_t)(kAcc - 1);
+                    const uint32_t acc_use = wt / (uint32_t)kAcc;
+                    const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
+                    if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 0, cta_t0);
+                    if (acc_use > 0 && !pre_acc) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status));
+                    if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 1, cta_t0);
+                    // Tile j reads pieces 0..j.  The transform warps finish pieces in order, so with
+                    // a transform piece j's barrier covers the earlier ones.  Without one the copies
+                    // land in any order: this issuer waits for pieces j-1 and j (its previous tile
+                    // of the group, j-2, waited for the two before).
+                    const uint32_t ops_bar = smem_u32(MODE == SPARQ_MODE_NONE ? &bar_win_full[b * kMaxG + j] : &bar_win_xf[b * kMaxG + j]);
+                    if (!pre_ops) {
+                        if (MODE == SPARQ_MODE_NONE && j > 0) SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar - 8u, wph, abort_flag, g.status));
+                        SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar, wph, abort_flag, g.status));
+                    }
+                    tc_fence_after();
+                    pre_acc = pre_ops = 0;
+                    const uint32_t step = (uint32_t)g.issuers;          // this issuer's next tile is number wt + step
+                    const bool look_ahead = j + (int)step < (int)walk.cnt;
+                    auto look = [&]() {
+                        if (!look_ahead) return;
+                        // a stage's first use needs no wait (the piece barrier stands in for it in the look)
+                        const uint32_t nacc = (wt + step) & (uint32_t)(kAcc - 1), nuse = (wt + step) / (uint32_t)kAcc;
+                        const uint32_t m = mbar_test3(nuse ? smem_u32(&bar_acc_empty[nacc]) : ops_bar, nuse ? (nuse - 1u) & 1u : wph,
+                                                      ops_bar + 8u, wph, ops_bar + 8u * step, wph);
+                        pre_acc = nuse ? (m & 1u) : 1u;
+                        pre_ops = (MODE == SPARQ_MODE_NONE) ? (uint32_t)((m & 6u) == 6u) : (m >> 2);
+                    };
+                    const uint64_t a_desc0 = a_grp + (uint64_t)((uint32_t)j * tile16);
+                    const long long is0 = SPARQ_PROF_NOW();
+                    if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 2, cta_t0);
+                    // One (tap, channel block) of the tile: wait for its weights when they are
+                    // streamed, then CB / 32 MMAs.  The descriptors are sums of warp-uniform
+                    // loop-carried values (no table, no division), so the address arithmetic of
+                    // consecutive MMAs is a couple of adds.
+                    auto issue_block = [&](const bool first, const uint32_t slot, const uint64_t adesc) {
+                        uint64_t bdesc;
+                        if (B_RESIDENT) {
+                            bdesc = b_desc0 + (uint64_t)(slot * (uint32_t)(kBBlock >> 4));
+                        } else {
+                            SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status));
+                            tc_fence_after();
+                            bdesc = b_desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kBBlock >> 4));
+                        }
+#pragma unroll
+                        for (int k = 0; k < CB / 32; ++k)
+                            tc_mma_i8_if(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
+                                         (!first || k > 0) ? 1u : 0u, elected);
+                        if (!B_RESIDENT) {
+                            tc_commit_if(smem_u32(&bar_b_empty[s]), elected);
+                            if (++s == g.b_stages) { s = 0; bph ^= 1u; }
+                        }
+                    };
+                    // channel block outer, tap inner; the resident slot of (tap, cb) is tap * c_blocks + cb
+                    uint64_t a_cb = a_desc0;
+                    const uint32_t cbs = (uint32_t)g.c_blocks;
+                    if (g.R == 3 && g.S == 3) {
+                        for (uint32_t cb = 0; cb < cbs; ++cb, a_cb += plane16) {
+#pragma unroll
+                            for (int r = 0; r < 3; ++r) {
+#pragma unroll
+                                for (int sx = 0; sx < 3; ++sx)
+                                    issue_block(cb == 0 && r == 0 && sx == 0, (uint32_t)(r * 3 + sx) * cbs + cb,
+                                                a_cb + (uint64_t)((uint32_t)r * row16 + (uint32_t)(sx * (CB >> 4))));
+                                if (r == 0 && cb == 0) look();
+                            }
+                        }
                     } else {
-                        SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status));
-                        tc_fence_after();
-                        bdesc = b_desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kBBlock >> 4));
+                        for (uint32_t cb = 0; cb < cbs; ++cb, a_cb += plane16) {
+                            uint64_t a_r = a_cb;
+                            uint32_t slot = cb;
+                            for (int r = 0; r < g.R; ++r, a_r += row16) {
+                                for (int sx = 0; sx < g.S; ++sx, slot += cbs)
+                                    issue_block(cb == 0 && r == 0 && sx == 0, slot, a_r + (uint64_t)(uint32_t)(sx * (CB >> 4)));
+                                if (r == 0 && cb == 0) look();
+                            }
+                        }
                     }
-#pragma unroll
-                    for (int k = 0; k < CB / 32; ++k)
-                        tc_mma_i8_if(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
-                                     (kb > 0 || k > 0) ? 1u : 0u, elected);
-                    if (!B_RESIDENT) {
-                        tc_commit_if(smem_u32(&bar_b_empty[s]), elected);
-                        if (++s == g.b_stages) { s = 0; bph ^= 1u; }
-                    }
-                };
-                uint32_t kb = 0;
-                uint64_t a_cb = a_desc0;
-                if (g.R == 3 && g.S == 3) {
-                    for (int cb = 0; cb < g.c_blocks; ++cb, a_cb += plane16) {
-#pragma unroll
-                        for (int r = 0; r < 3; ++r)
-#pragma unroll
-                            for (int sx = 0; sx < 3; ++sx, ++kb)
-                                issue_block(kb, a_cb + (uint64_t)((uint32_t)r * row16 + (uint32_t)(sx * (CB >> 4))));
-                    }
-                } else {
-                    for (int cb = 0; cb < g.c_blocks; ++cb, a_cb += plane16) {
-                        uint64_t a_r = a_cb;
-                        for (int r = 0; r < g.R; ++r, a_r += row16)
-                            for (int sx = 0; sx < g.S; ++sx, ++kb)
-                                issue_block(kb, a_r + (uint64_t)(uint32_t)(sx * (CB >> 4)));
-                    }
+                    mi += SPARQ_PROF_NOW() - is0;
+                    if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 3, cta_t0);
+                    tc_commit_if(smem_u32(&bar_acc_full[acc]), elected);      // accumulator complete
+                    if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 4, cta_t0);
                 }
-                mi += SPARQ_PROF_NOW() - is0;
-                tc_commit_if(smem_u32(&bar_win_empty[b]), elected);       // window reusable once these MMAs retire
-                tc_commit_if(smem_u32(&bar_acc_full[acc]), elected);      // accumulator complete
-                if (++b == g.win_bufs) { b = 0; wph ^= 1u; }
+                // The buffer goes back to the producer once both issuers have arrived and their
+                // MMAs have retired.  With a transform, first make sure that every transform warp
+                // is past all of this use's barriers (they arrive on the last piece's barrier
+                // last), so that none of them can still be waiting on a phase when the producer
+                // starts the next.
+                if (MODE != SPARQ_MODE_NONE && (int)walk.cnt < g.G)
+                    SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b * kMaxG + g.G - 1]), wph, abort_flag, g.status));
+                if (issued) {
+                    tc_commit_if(smem_u32(&bar_win_empty[b]), elected);
+                } else {
+                    // No tile of this group was this issuer's.  It arrives only once the producer has
+                    // started this use of the buffer (its first piece has landed), i.e. after the
+                    // previous use's phase of the barrier has completed.
+                    mbar_wait(smem_u32(&bar_win_full[b * kMaxG]), wph, abort_flag, g.status);
+                    if (elected) mbar_arrive(smem_u32(&bar_win_empty[b]));
+                }
+                ++gi;
             }
-            SPARQ_PROF_STORE(2, mw);
-            SPARQ_PROF_STORE(3, ma);
-            SPARQ_PROF_STORE(11, mb);
-            SPARQ_PROF_STORE(12, mi);
-            SPARQ_PROF_STORE(4, SPARQ_PROF_NOW() - mt0);
+            if (me == 0) {
+                SPARQ_PROF_STORE(2, mw);
+                SPARQ_PROF_STORE(3, ma);
+                SPARQ_PROF_STORE(11, mb);
+                SPARQ_PROF_STORE(12, mi);
+                SPARQ_PROF_STORE(4, SPARQ_PROF_NOW() - mt0);
+            }
+            // all tensor-core work of this CTA has retired before tensor memory is freed
             tc_commit_if(smem_u32(&bar_done), elected);
             mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, true);
+            if (me == 0) SPARQ_PROF_TL(0, 40, cta_t0);
         }
         __syncwarp();
     } else if (warp < kFirstEpiWarp + epi_warps(MODE)) {
@@ -315,17 +497,17 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 rs[i] = s_scale[cbase + i];
                 rb[i] = s_bias[cbase + i];
             }
-            const uint32_t tiles32 = (uint32_t)total_tiles, tpi = (uint32_t)g.tiles_per_img;
-            for (uint32_t tile = blockIdx.x; tile < tiles32; tile += gridDim.x, ++wt) {
-                const uint32_t acc = wt & 1u;
+            while (walk.next()) {
+              for (int j = 0; j < (int)walk.cnt; ++j, ++wt) {
+                const uint32_t acc = wt & (uint32_t)(kAcc - 1);
                 // coordinates first: they do not depend on the accumulator
-                const uint32_t img = tile / tpi;
-                const int oh = (int)(tile - img * tpi) * g.TR + tr;
+                const int oh = ((int)walk.tin + j) * g.TR + tr;
                 const bool row_ok = slot_ok && (oh < g.Ho);
-                uint8_t *dst = g.u8_out + (((int64_t)img * g.Ho + oh) * g.Wo + ow) * 64 + cbase;
+                uint8_t *dst = g.u8_out + (((int64_t)walk.img * g.Ho + oh) * g.Wo + ow) * 64 + cbase;
                 const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + (uint32_t)cbase;
-                SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt >> 1) & 1u, abort_flag, g.status));
+                SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status));
                 tc_fence_after();
+                if (warp == kFirstEpiWarp && lane == 0) SPARQ_PROF_TL(1, 2 * wt, cta_t0);
 #pragma unroll
                 for (int hh = 0; hh < kColsPerWarp / 16; ++hh) {
                     uint32_t v[16];
@@ -340,99 +522,98 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                     uint32_t w[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        uint32_t b[4];
+                        uint32_t bb[4];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int c = hh * 16 + 4 * q + j;
-                            const float y = ev.small_acc ? dequant<true>((int32_t)v[4 * q + j], rs[c], rb[c], ev.relu_op)
-                                                         : dequant<false>((int32_t)v[4 * q + j], rs[c], rb[c], ev.relu_op);
-                            b[j] = requant_bits(y, ev.inv_out_scale);
+                        for (int jj = 0; jj < 4; ++jj) {
+                            const int c = hh * 16 + 4 * q + jj;
+                            const float y = ev.small_acc ? dequant<true>((int32_t)v[4 * q + jj], rs[c], rb[c], ev.relu_op)
+                                                         : dequant<false>((int32_t)v[4 * q + jj], rs[c], rb[c], ev.relu_op);
+                            bb[jj] = requant_bits(y, ev.inv_out_scale);
                         }
-                        w[q] = pack4(b[0], b[1], b[2], b[3]);
+                        w[q] = pack4(bb[0], bb[1], bb[2], bb[3]);
                     }
-                    if (ev.next_mode != SPARQ_MODE_NONE) {
-                        const bool fast4 = ev.next_xf.n == 4 && ev.next_xf.rounds == 0;
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            if (ev.next_mode == SPARQ_MODE_VSPARQ) {
-                                if (fast4) w[q] = ev.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 4, true, false>(w[q], ev.next_xf)
-                                                              : xform_word<SPARQ_MODE_VSPARQ, 4, false, false>(w[q], ev.next_xf);
-                                else w[q] = ev.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 0, true, true>(w[q], ev.next_xf)
-                                                        : xform_word<SPARQ_MODE_VSPARQ, 0, false, true>(w[q], ev.next_xf);
-                            } else {
-                                if (fast4) w[q] = ev.next_rnd ? xform_word<SPARQ_MODE_BSPARQ, 4, true, false>(w[q], ev.next_xf)
-                                                              : xform_word<SPARQ_MODE_BSPARQ, 4, false, false>(w[q], ev.next_xf);
-                                else w[q] = ev.next_rnd ? xform_word<SPARQ_MODE_BSPARQ, 0, true, true>(w[q], ev.next_xf)
-                                                        : xform_word<SPARQ_MODE_BSPARQ, 0, false, true>(w[q], ev.next_xf);
-                            }
-                        }
-                    }
+                    if (ev.next_mode != SPARQ_MODE_NONE) next_xform_words(w, 4, ev.next_mode, ev.next_rnd, ev.next_xf);
                     *reinterpret_cast<uint4 *>(dst + hh * 16) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
+                if (warp == kFirstEpiWarp && lane == 0) SPARQ_PROF_TL(1, 2 * wt + 1, cta_t0);
+              }
             }
         } else
-        for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
-            const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
-            const int acc = wt & 1;
-            const uint32_t acc_use = wt >> 1;
+        while (walk.next()) {
+          for (int j = 0; j < (int)walk.cnt; ++j, ++wt) {
+            const int64_t nt = (int64_t)walk.nt;
+            const int acc = (int)(wt & (uint32_t)(kAcc - 1));
+            const uint32_t acc_use = wt / (uint32_t)kAcc;
             if (ev.need_f && nt != staged_nt) {
                 staged_nt = nt;
                 epi_stage_scale_bias<kEpi>(g, nt * BN, BN, et, s_scale, s_bias);
             }
             SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status));
             tc_fence_after();
-            const int img = (int)(mt / g.tiles_per_img);
-            const int oh = (int)(mt % g.tiles_per_img) * g.TR + tr;
+            const int oh = ((int)walk.tin + j) * g.TR + tr;
             const bool row_ok = slot_ok && (oh < g.Ho);
-            const int64_t row = ((int64_t)img * g.Ho + oh) * g.Wo + ow;
+            const int64_t row = ((int64_t)walk.img * g.Ho + oh) * g.Wo + ow;
             const int cbase = part * kColsPerWarp;
             const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + cbase);
             epi_warp_columns<kColsPerWarp>(ev, taddr0, cbase, row, row_ok, nt * BN, s_scale, s_bias,
                                       smem_u32(&bar_acc_empty[acc]), lane);
+          }
         }
         if (warp == kFirstEpiWarp && lane == 0) {
             SPARQ_PROF_STORE(5, ew);
             SPARQ_PROF_STORE(6, SPARQ_PROF_NOW() - et0);
         }
     } else if (MODE != SPARQ_MODE_NONE) {
-        // ================= transform: once per window =================
-        const int xt = threadIdx.x - kFirstXfWarp * 32;
-        constexpr int kXfThreads = kNumXfWarps * 32;
+        // ================= transform: once per piece =================
+        const uint32_t xt = threadIdx.x - kFirstXfWarp * 32;
+        constexpr uint32_t kXfThreads = kNumXfWarps * 32;
         const XformDev xf = g.xf;
-        // whole groups of kXfThreads * 4 vectors; the tail group runs into the plane's slack
-        // rows, which no valid output reads (the host sizes the plane for it)
-        const int groups = (g.box_bytes + kXfThreads * 64 - 1) / (kXfThreads * 64);
-        uint32_t wt = 0;
+        uint32_t gi = 0;
         long long xw = 0;
         const long long xt0 = SPARQ_PROF_NOW();
-        for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++wt) {
-            const int b = wt % g.win_bufs;
-            SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_win_full[b]), (wt / g.win_bufs) & 1, abort_flag, g.status));
-            for (int cb = 0; cb < g.c_blocks; ++cb) {
-                const uint32_t base = win_buf(b) + (uint32_t)cb * g.plane_bytes + (uint32_t)xt * 16u;
-                for (int grp = 0; grp < groups; ++grp) {
-                    const uint32_t gbase = base + (uint32_t)grp * (kXfThreads * 64);
-                    uint4 v[4];
+        while (walk.next()) {
+            const int b = gi % g.win_bufs;
+            const uint32_t wph = (gi / g.win_bufs) & 1u;
+            for (int j = 0; j < g.G; ++j) {
+                SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), wph, abort_flag, g.status));
+                if (warp == kFirstXfWarp && lane == 0 && gi == 0) SPARQ_PROF_TL(2, 2 * j, cta_t0);
+                if (j < (int)walk.cnt) {
+                    const uint32_t nvec = piece_len(j) >> 4;
+                    uint32_t pbase = win_buf(b) + piece_off(j);
+                    for (int cb = 0; cb < g.c_blocks; ++cb, pbase += (uint32_t)g.plane_bytes) {
+                        // four independent 16-byte vectors per thread and step; the last step of a
+                        // piece may be short
+                        for (uint32_t v0 = xt; v0 < nvec; v0 += 4 * kXfThreads) {
+                            uint4 v[4];
+                            bool ok[4];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                                     : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w)
-                                     : "r"(gbase + (uint32_t)(j * kXfThreads * 16)));
+                            for (int q = 0; q < 4; ++q) {
+                                ok[q] = v0 + (uint32_t)q * kXfThreads < nvec;
+                                if (ok[q])
+                                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                                 : "=r"(v[q].x), "=r"(v[q].y), "=r"(v[q].z), "=r"(v[q].w)
+                                                 : "r"(pbase + (v0 + (uint32_t)q * kXfThreads) * 16u));
+                            }
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        v[j].x = xform_word<MODE, XN, RND, XN == 0>(v[j].x, xf);
-                        v[j].y = xform_word<MODE, XN, RND, XN == 0>(v[j].y, xf);
-                        v[j].z = xform_word<MODE, XN, RND, XN == 0>(v[j].z, xf);
-                        v[j].w = xform_word<MODE, XN, RND, XN == 0>(v[j].w, xf);
-                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
-                                     :: "r"(gbase + (uint32_t)(j * kXfThreads * 16)),
-                                        "r"(v[j].x), "r"(v[j].y), "r"(v[j].z), "r"(v[j].w) : "memory");
+                            for (int q = 0; q < 4; ++q) {
+                                if (!ok[q]) continue;
+                                v[q].x = xform_word<MODE, XN, RND, XN == 0>(v[q].x, xf);
+                                v[q].y = xform_word<MODE, XN, RND, XN == 0>(v[q].y, xf);
+                                v[q].z = xform_word<MODE, XN, RND, XN == 0>(v[q].z, xf);
+                                v[q].w = xform_word<MODE, XN, RND, XN == 0>(v[q].w, xf);
+                                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
+                                             :: "r"(pbase + (v0 + (uint32_t)q * kXfThreads) * 16u),
+                                                "r"(v[q].x), "r"(v[q].y), "r"(v[q].z), "r"(v[q].w) : "memory");
+                            }
+                        }
                     }
+                    fence_proxy_async_smem();
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_win_xf[b * kMaxG + j]));
+                if (warp == kFirstXfWarp && lane == 0 && gi == 0) SPARQ_PROF_TL(2, 2 * j + 1, cta_t0);
             }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bar_win_xf[b]));
+            ++gi;
         }
         if (warp == kFirstXfWarp && lane == 0) {
             SPARQ_PROF_STORE(7, xw);
@@ -442,7 +623,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
 
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) SPARQ_PROF_STORE(10, SPARQ_PROF_NOW() - cta_t0);
+    if (threadIdx.x == 0) { SPARQ_PROF_STORE(10, SPARQ_PROF_NOW() - cta_t0); SPARQ_PROF_TL(3, 0, cta_t0); }
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
@@ -451,7 +632,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
 }
 
 template <int BN, int CB, bool B_RESIDENT>
-cudaError_t launch_window_shape(const CUtensorMap &mx, const CUtensorMap &mw, const WindowArgs &g,
+cudaError_t launch_window_shape(const CUtensorMap &mx0, const CUtensorMap &mx1, const CUtensorMap &mw, const WindowArgs &g,
                                 int mode, int n, int rnd, int grid, int smem_bytes, cudaStream_t st);
 
 #define SPARQ_LAUNCH_WINDOW_VARIANT(MODE_, XN_, RND_)                                                  \
@@ -467,12 +648,13 @@ cudaError_t launch_window_shape(const CUtensorMap &mx, const CUtensorMap &mw, co
             if (e_ != cudaSuccess) return e_;                                                          \
             if (dev_ >= 0 && dev_ < 64) attr_set[dev_] = true;                                         \
         }                                                                                              \
-        return launch_pdl(kfn, grid, smem_bytes, st, mx, mw, g);                                       \
+        return launch_pdl<kWindowThreads>(kfn, grid, smem_bytes, st, mx0, mx1, mw, g);                                       \
     } while (0)
 
 #define SPARQ_DEFINE_WINDOW_SHAPE(BN_, CB_, RES_)                                                      \
     template <>                                                                                        \
-    cudaError_t launch_window_shape<BN_, CB_, RES_>(const CUtensorMap &mx, const CUtensorMap &mw,      \
+    cudaError_t launch_window_shape<BN_, CB_, RES_>(const CUtensorMap &mx0, const CUtensorMap &mx1,    \
+                                                    const CUtensorMap &mw,                             \
                                                     const WindowArgs &g, int mode, int n, int rnd,     \
                                                     int grid, int smem_bytes, cudaStream_t st)         \
     {                                                                                                  \

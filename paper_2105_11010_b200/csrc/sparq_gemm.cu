@@ -2,6 +2,7 @@
 // (tiled for the GEMM view, im2col for the convolution), launch.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <cstring>
 
 #include "sparq_conv_window_kernel.cuh"
@@ -10,6 +11,7 @@ namespace sparq {
 
 #ifdef SPARQ_PROF
 __device__ long long g_prof[148 * 16];
+__device__ long long g_prof_tl[4 * 64];
 #endif
 
 void release_gemm_state() {}
@@ -239,6 +241,22 @@ static int encode_window(CUtensorMap *map, const void *ptr, int n, int h, int w,
     return SPARQ_OK;
 }
 
+// Weights [cout][K] seen as (cb bytes, cout rows, K / cb blocks): one box brings every
+// (tap, channel block) of bn filters into consecutive bn x cb shared-memory blocks.
+// Returns the driver's result; the caller falls back to one copy per block if it is refused.
+static CUresult encode_weight_blocks(CUtensorMap *map, const void *ptr, int64_t K, int cout, int cb, int bn, int blocks)
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn && driver_fn("cuTensorMapEncodeTiled", (void **)&fn) != SPARQ_OK) return CUDA_ERROR_NOT_FOUND;
+    cuuint64_t dims[3] = {(cuuint64_t)cb, (cuuint64_t)cout, (cuuint64_t)blocks};
+    cuuint64_t strides[2] = {(cuuint64_t)K, (cuuint64_t)cb};
+    cuuint32_t box[3] = {(cuuint32_t)cb, (cuuint32_t)bn, (cuuint32_t)blocks};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(cb), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
 constexpr int kMaxDynSmem = kWindowMaxDynSmem;
 
 // Stride-1 filters larger than 1x1: the window kernel, when its tiling fits.  Returns
@@ -257,13 +275,6 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     const int c_blocks = c / cb;
     const int taps = r * s;
     const int kb_count = taps * c_blocks;
-    const int rows_alloc = (r - 1) * wp + (s - 1) + 128;
-    // a plane holds every row the MMA may touch and the whole 16 KB groups the transform rewrites
-    const int box_bytes = cb * wp * (tr + r - 1);
-    int plane_bytes = rows_alloc * cb;
-    if (plane_bytes < (box_bytes + 16383) / 16384 * 16384) plane_bytes = (box_bytes + 16383) / 16384 * 16384;
-    plane_bytes = (plane_bytes + 1023) / 1024 * 1024;
-    const int win_bytes = plane_bytes * c_blocks;
     const int tiles_per_img = (ho + tr - 1) / tr;
     const int64_t m_tiles = (int64_t)n * tiles_per_img;
 
@@ -277,40 +288,85 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     }
     const int b_block = bn * cb;
     const int n_tiles = (cout + bn - 1) / bn;
+    const int64_t units = m_tiles * n_tiles;
+    if (units >= (int64_t)1 << 31) return 0;
+    const int grid = (int)(units < sms ? units : sms);
+
+    // Shared memory of one window buffer when up to `grp` tiles share it: a plane (one channel
+    // block) holds every row the MMA of the group's last tile may touch.
+    auto plane_for = [&](int grp) {
+        const int rows_alloc = (grp - 1) * tr * wp + (r - 1) * wp + (s - 1) + 128;
+        return (rows_alloc * cb + 1023) / 1024 * 1024;
+    };
+    // Tiles per group: with one column tile, as many as a CTA's share of the tile sequence
+    // has (more would never be used) while two window buffers still fit beside the weights.
+    // A later piece must land on a 128-byte boundary (TMA destination alignment).
+    int gmax = 1;
+    if (n_tiles == 1) {
+        gmax = (int)((units + grid - 1) / grid);
+        if (gmax > tiles_per_img) gmax = tiles_per_img;
+        if (gmax > kMaxG) gmax = kMaxG;
+        if (cb == 64 && (((tr * wp) & 1) || (((r - 1) * wp) & 1))) gmax = 1;
+    }
     bool resident = false;
-    int win_bufs = 2, b_stages = 0;
-    if (bn != 256 && n_tiles == 1 && 1024 + 2 * win_bytes + kb_count * b_block <= kMaxDynSmem) {
+    int win_bufs = 2, b_stages = 0, grp = 1;
+    if (bn != 256 && n_tiles == 1 && 1024 + 2 * plane_for(1) * c_blocks + kb_count * b_block <= kMaxDynSmem) {
         resident = true;
         b_stages = kb_count;
-        while (win_bufs < kMaxWinBufs && 1024 + (win_bufs + 1) * win_bytes + kb_count * b_block <= kMaxDynSmem) ++win_bufs;
+        grp = gmax;
+        while (grp > 1 && 1024 + 2 * plane_for(grp) * c_blocks + kb_count * b_block > kMaxDynSmem) --grp;
+        // more buffers only help while a CTA has more groups than buffers
+        const int groups_per_cta = (int)((units + grid - 1) / grid + grp - 1) / grp + 1;
+        while (win_bufs < kMaxWinBufs && win_bufs < groups_per_cta &&
+               1024 + (win_bufs + 1) * plane_for(grp) * c_blocks + kb_count * b_block <= kMaxDynSmem) ++win_bufs;
     } else {
         if (bn == 64) return 0;                          // only the resident form is built for 64-wide tiles
-        const int left = kMaxDynSmem - 1024 - 2 * win_bytes;
+        grp = gmax;
+        while (grp > 1 && kMaxDynSmem - 1024 - 2 * plane_for(grp) * c_blocks < 4 * b_block) --grp;
+        const int win_bytes1 = plane_for(grp) * c_blocks;
+        const int left = kMaxDynSmem - 1024 - 2 * win_bytes1;
         b_stages = left / b_block;
         if (b_stages > kMaxBStages) b_stages = kMaxBStages;
         if (b_stages < 2) return 0;
         // spare room beyond four weight stages goes to a third window buffer
-        if (b_stages > 4 && 1024 + 3 * win_bytes + 4 * b_block <= kMaxDynSmem) {
+        if (b_stages > 4 && 1024 + 3 * win_bytes1 + 4 * b_block <= kMaxDynSmem) {
             win_bufs = 3;
-            b_stages = (kMaxDynSmem - 1024 - 3 * win_bytes) / b_block;
+            b_stages = (kMaxDynSmem - 1024 - 3 * win_bytes1) / b_block;
             if (b_stages > kMaxBStages) b_stages = kMaxBStages;
         }
     }
+    const int plane_bytes = plane_for(grp);
+    const int win_bytes = plane_bytes * c_blocks;
     const int smem_bytes = 1024 + win_bufs * win_bytes + b_stages * b_block;
 
-    CUtensorMap mx, mw;
+    CUtensorMap mx, mx1, mw;
     int rc = encode_window(&mx, x_in, n, h, w, c, cb, wp, tr + r - 1);
     if (rc != SPARQ_OK) return rc;
-    const int64_t K = (int64_t)r * s * c;
-    rc = encode_2d(&mw, wgt, K, cout, K, cb, bn);
+    rc = encode_window(&mx1, x_in, n, h, w, c, cb, wp, tr);
     if (rc != SPARQ_OK) return rc;
+    const int64_t K = (int64_t)r * s * c;
+    bool w_one_copy = resident && kb_count <= 256 &&
+                      encode_weight_blocks(&mw, wgt, K, cout, cb, bn, kb_count) == CUDA_SUCCESS;
+    if (!w_one_copy) {
+        rc = encode_2d(&mw, wgt, K, cout, K, cb, bn);
+        if (rc != SPARQ_OK) return rc;
+    }
 
     WindowArgs g;
     memset(&g, 0, sizeof(g));
+    g.w_one_copy = w_one_copy ? 1 : 0;
+    g.issuers = 2;
+#if defined(SPARQ_PROF) || defined(SPARQ_TUNE)
+    if (const char *ev = getenv("SPARQ_ISSUERS")) g.issuers = atoi(ev) == 1 ? 1 : 2;
+#endif
     g.N = cout; g.K = K;
     g.n_img = n; g.H = h; g.W = w; g.C = c; g.R = r; g.S = s; g.pad_h = pad_h; g.pad_w = pad_w; g.Ho = ho; g.Wo = wo;
     g.Wp = wp; g.TR = tr; g.tiles_per_img = tiles_per_img; g.c_blocks = c_blocks;
-    g.box_bytes = box_bytes;
+    g.G = grp;
+    g.piece0_bytes = cb * wp * (tr + r - 1);
+    g.piece_bytes = cb * wp * tr;
+    g.n_tiles = (uint32_t)n_tiles;
+    g.units = (uint32_t)units;
     g.plane_bytes = plane_bytes;
     g.win_bufs = win_bufs;
     g.b_stages = b_stages;
@@ -322,13 +378,11 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     g.residual_scale = e->residual_scale;
     rc = next_transform_args(e, g.N, &g.next_mode, &g.next_rnd, &g.next_xf);
     if (rc != SPARQ_OK) return rc;
-    const int64_t tiles = m_tiles * n_tiles;
-    const int grid = (int)(tiles < sms ? tiles : sms);
     cudaError_t ce;
-    if (bn == 64) ce = launch_window_shape<64, 64, true>(mx, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
-    else if (bn == 128 && resident) ce = launch_window_shape<128, 128, true>(mx, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
-    else if (bn == 128) ce = launch_window_shape<128, 128, false>(mx, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
-    else ce = launch_window_shape<256, 128, false>(mx, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
+    if (bn == 64) ce = launch_window_shape<64, 64, true>(mx, mx1, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
+    else if (bn == 128 && resident) ce = launch_window_shape<128, 128, true>(mx, mx1, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
+    else if (bn == 128) ce = launch_window_shape<128, 128, false>(mx, mx1, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
+    else ce = launch_window_shape<256, 128, false>(mx, mx1, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
     if (ce != cudaSuccess) return cuda_error(ce, "sparq_conv_window_kernel launch");
     return 1;
 }
@@ -460,5 +514,9 @@ extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, in
 extern "C" __attribute__((visibility("default"))) int sparq_prof_read(long long *out)
 {
     return (int)cudaMemcpyFromSymbol(out, sparq::g_prof, sizeof(long long) * 148 * 16);
+}
+extern "C" __attribute__((visibility("default"))) int sparq_prof_read_timeline(long long *out)
+{
+    return (int)cudaMemcpyFromSymbol(out, sparq::g_prof_tl, sizeof(long long) * 4 * 64);
 }
 #endif

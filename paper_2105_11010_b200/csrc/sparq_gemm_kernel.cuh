@@ -48,7 +48,10 @@ constexpr long long kWaitLimitCycles = 2000000000LL;
 extern __device__ long long g_prof[148 * 16];
 #define SPARQ_PROF_NOW() clock64()
 #define SPARQ_PROF_STORE(slot, v) (g_prof[blockIdx.x * 16 + (slot)] = (v))
+extern __device__ long long g_prof_tl[4 * 64];      // CTA 0's timeline: [role][event]
+#define SPARQ_PROF_TL(role, idx, t0) do { if (blockIdx.x == 0 && (idx) < 64) g_prof_tl[(role) * 64 + (idx)] = clock64() - (t0); } while (0)
 #else
+#define SPARQ_PROF_TL(role, idx, t0) ((void)0)
 #define SPARQ_PROF_NOW() 0LL
 #define SPARQ_PROF_STORE(slot, v) ((void)(v))
 #endif
@@ -117,6 +120,39 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
+}
+
+// Non-blocking look at a phase: 1 if it has completed.  Unlike try_wait this never suspends
+// the thread, and nothing waits for its result until the value is used.
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+
+// Three looks at once (bit i: barrier i): all reads are in flight together before any answer
+// is consumed.
+__device__ __forceinline__ uint32_t mbar_test3(uint32_t bar0, uint32_t parity0, uint32_t bar1, uint32_t parity1,
+                                               uint32_t bar2, uint32_t parity2)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p, q, r;\n\t.reg .u32 a, b, c;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 q, [%3], %4;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 r, [%5], %6;\n\t"
+        "selp.u32 a, 1, 0, p;\n\t"
+        "selp.u32 b, 2, 0, q;\n\t"
+        "selp.u32 c, 4, 0, r;\n\t"
+        "or.b32 a, a, b;\n\t"
+        "or.b32 %0, a, c;\n\t}"
+        : "=r"(ok) : "r"(bar0), "r"(parity0), "r"(bar1), "r"(parity1), "r"(bar2), "r"(parity2) : "memory");
+    return ok;
 }
 
 // Bounded wait.  Returns false (after flagging) if the phase did not complete in time or
@@ -318,6 +354,26 @@ __device__ __forceinline__ uint32_t pack4(uint32_t a, uint32_t b, uint32_t c, ui
     return prmt(prmt(a, b, 0x0040u), prmt(c, d, 0x0040u), 0x5410u);
 }
 
+// The next layer's transform on requantized bytes (producer-side SPARQ): four adjacent output
+// channels per word, pairs (2j, 2j+1) inside it.  Kept out of line: the epilogue loops are hot
+// and every variant inlined at every use made the kernels several times larger than the
+// instruction caches, which the warp roles share.
+static __device__ __noinline__ void next_xform_words(uint32_t *w, int count, int mode, int rnd, XformDev xf)
+{
+    const bool fast4 = xf.n == 4 && xf.rounds == 0;   // n = 4, all five placements
+    for (int q = 0; q < count; ++q) {
+        uint32_t x = w[q];
+        if (mode == SPARQ_MODE_VSPARQ) {
+            if (fast4) x = rnd ? xform_word<SPARQ_MODE_VSPARQ, 4, true, false>(x, xf) : xform_word<SPARQ_MODE_VSPARQ, 4, false, false>(x, xf);
+            else x = rnd ? xform_word<SPARQ_MODE_VSPARQ, 0, true, true>(x, xf) : xform_word<SPARQ_MODE_VSPARQ, 0, false, true>(x, xf);
+        } else {
+            if (fast4) x = rnd ? xform_word<SPARQ_MODE_BSPARQ, 4, true, false>(x, xf) : xform_word<SPARQ_MODE_BSPARQ, 4, false, false>(x, xf);
+            else x = rnd ? xform_word<SPARQ_MODE_BSPARQ, 0, true, true>(x, xf) : xform_word<SPARQ_MODE_BSPARQ, 0, false, true>(x, xf);
+        }
+        w[q] = x;
+    }
+}
+
 // Per-thread view of the epilogue's outputs and constants.
 struct EpiView {
     int64_t N;
@@ -458,25 +514,7 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[NV], i
                          requant_bits(__uint_as_float(v[4 * q + 1]), e.inv_out_scale),
                          requant_bits(__uint_as_float(v[4 * q + 2]), e.inv_out_scale),
                          requant_bits(__uint_as_float(v[4 * q + 3]), e.inv_out_scale));
-        if (e.next_mode != SPARQ_MODE_NONE) {
-            // the next layer's transform on the bytes just produced: four adjacent output
-            // channels per word, pairs (2j, 2j+1) inside it
-            const bool fast4 = e.next_xf.n == 4 && e.next_xf.rounds == 0;   // n = 4, all five placements
-#pragma unroll
-            for (int q = 0; q < NQ; ++q) {
-                if (e.next_mode == SPARQ_MODE_VSPARQ) {
-                    if (fast4) w[q] = e.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 4, true, false>(w[q], e.next_xf)
-                                                 : xform_word<SPARQ_MODE_VSPARQ, 4, false, false>(w[q], e.next_xf);
-                    else w[q] = e.next_rnd ? xform_word<SPARQ_MODE_VSPARQ, 0, true, true>(w[q], e.next_xf)
-                                           : xform_word<SPARQ_MODE_VSPARQ, 0, false, true>(w[q], e.next_xf);
-                } else {
-                    if (fast4) w[q] = e.next_rnd ? xform_word<SPARQ_MODE_BSPARQ, 4, true, false>(w[q], e.next_xf)
-                                                 : xform_word<SPARQ_MODE_BSPARQ, 4, false, false>(w[q], e.next_xf);
-                    else w[q] = e.next_rnd ? xform_word<SPARQ_MODE_BSPARQ, 0, true, true>(w[q], e.next_xf)
-                                           : xform_word<SPARQ_MODE_BSPARQ, 0, false, true>(w[q], e.next_xf);
-                }
-            }
-        }
+        if (e.next_mode != SPARQ_MODE_NONE) next_xform_words(w, NQ, e.next_mode, e.next_rnd, e.next_xf);
         if (full) {
             if constexpr (NV == 32) {
                 if (e.u8_wide) {
@@ -796,13 +834,12 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 }
 
 // Launch with programmatic stream serialization allowed (see dep_wait / dep_launch).
-template <class Kernel, class Args>
-cudaError_t launch_pdl(Kernel kfn, int grid, int smem_bytes, cudaStream_t st, const CUtensorMap &m0,
-                       const CUtensorMap &m1, const Args &g)
+template <int THREADS = kGemmThreads, class Kernel, class... KernelArgs>
+cudaError_t launch_pdl(Kernel kfn, int grid, int smem_bytes, cudaStream_t st, const KernelArgs &...args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(kGemmThreads);
+    cfg.blockDim = dim3(THREADS);
     cfg.dynamicSmemBytes = (size_t)smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -810,7 +847,7 @@ cudaError_t launch_pdl(Kernel kfn, int grid, int smem_bytes, cudaStream_t st, co
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kfn, m0, m1, g);
+    return cudaLaunchKernelEx(&cfg, kfn, args...);
 }
 
 // Host launcher for one tile shape; picks the transform variant.  Defined once per
