@@ -4,6 +4,7 @@
 
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 #include "sparq_conv_window_kernel.cuh"
 
@@ -37,6 +38,41 @@ static int driver_fn(const char *name, void **fn)
 
 static CUtensorMapSwizzle swizzle_for(int bk) { return bk == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B; }
 
+// A tensor map is a pure function of the arguments it is encoded from (address, extents,
+// strides, box, swizzle), and encoding one costs the host several microseconds -- as much as
+// a small layer takes on the device.  Networks call the same layers with the same buffers
+// over and over, so encoded maps are kept in a small direct-mapped table keyed by those
+// arguments.  Host memory only; nothing to release.
+struct MapKey {
+    uint64_t v[14];
+    bool operator==(const MapKey &o) const { return memcmp(v, o.v, sizeof(v)) == 0; }
+};
+struct MapSlot { bool used; MapKey key; CUtensorMap map; };
+constexpr int kMapSlots = 256;
+static MapSlot g_map_cache[kMapSlots];
+static std::mutex g_map_mutex;
+
+static unsigned map_hash(const MapKey &k)
+{
+    uint64_t h = 1469598103934665603ull;
+    for (uint64_t x : k.v) { h ^= x; h *= 1099511628211ull; h ^= h >> 29; }
+    return (unsigned)(h % kMapSlots);
+}
+static bool map_lookup(const MapKey &k, CUtensorMap *out)
+{
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    const MapSlot &s = g_map_cache[map_hash(k)];
+    if (!s.used || !(s.key == k)) return false;
+    *out = s.map;
+    return true;
+}
+static void map_store(const MapKey &k, const CUtensorMap &m)
+{
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    MapSlot &s = g_map_cache[map_hash(k)];
+    s.used = true; s.key = k; s.map = m;
+}
+
 // 2-D K-contiguous matrix [rows][K] with row pitch ld bytes; box = bk x box_rows.
 static int encode_2d(CUtensorMap *map, const void *ptr, int64_t K, int64_t rows, int64_t ld, int bk, int box_rows)
 {
@@ -45,6 +81,8 @@ static int encode_2d(CUtensorMap *map, const void *ptr, int64_t K, int64_t rows,
         int rc = driver_fn("cuTensorMapEncodeTiled", (void **)&fn);
         if (rc != SPARQ_OK) return rc;
     }
+    const MapKey key = {{1, (uint64_t)(uintptr_t)ptr, (uint64_t)K, (uint64_t)rows, (uint64_t)ld, (uint64_t)bk, (uint64_t)box_rows}};
+    if (map_lookup(key, map)) return SPARQ_OK;
     cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)ld};
     cuuint32_t box[2] = {(cuuint32_t)bk, (cuuint32_t)box_rows};
@@ -53,6 +91,7 @@ static int encode_2d(CUtensorMap *map, const void *ptr, int64_t K, int64_t rows,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(bk), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return set_error(SPARQ_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    map_store(key, *map);
     return SPARQ_OK;
 }
 
@@ -65,6 +104,9 @@ static int encode_im2col(CUtensorMap *map, const void *ptr, int n, int h, int w,
         int rc = driver_fn("cuTensorMapEncodeIm2col", (void **)&fn);
         if (rc != SPARQ_OK) return rc;
     }
+    const MapKey key = {{2, (uint64_t)(uintptr_t)ptr, (uint64_t)n, (uint64_t)h, (uint64_t)w, (uint64_t)c, (uint64_t)r, (uint64_t)s,
+                         (uint64_t)stride_h, (uint64_t)stride_w, (uint64_t)(int64_t)pad_h, (uint64_t)(int64_t)pad_w, (uint64_t)bk}};
+    if (map_lookup(key, map)) return SPARQ_OK;
     cuuint64_t dims[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
     cuuint64_t strides[3] = {(cuuint64_t)c, (cuuint64_t)c * w, (cuuint64_t)c * w * h};
     // Base pixels (the filter's top-left tap) run from -pad to dim - 1 + upper.
@@ -75,6 +117,7 @@ static int encode_im2col(CUtensorMap *map, const void *ptr, int n, int h, int w,
                       (cuuint32_t)bk, (cuuint32_t)kBM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(bk),
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (res != CUDA_SUCCESS) return set_error(SPARQ_ERR_CUDA, "cuTensorMapEncodeIm2col failed with CUresult %d", (int)res);
+    map_store(key, *map);
     return SPARQ_OK;
 }
 
@@ -230,6 +273,8 @@ static int encode_window(CUtensorMap *map, const void *ptr, int n, int h, int w,
         int rc = driver_fn("cuTensorMapEncodeTiled", (void **)&fn);
         if (rc != SPARQ_OK) return rc;
     }
+    const MapKey key = {{3, (uint64_t)(uintptr_t)ptr, (uint64_t)n, (uint64_t)h, (uint64_t)w, (uint64_t)c, (uint64_t)cb, (uint64_t)wp, (uint64_t)rows}};
+    if (map_lookup(key, map)) return SPARQ_OK;
     cuuint64_t dims[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
     cuuint64_t strides[3] = {(cuuint64_t)c, (cuuint64_t)c * w, (cuuint64_t)c * w * h};
     cuuint32_t box[4] = {(cuuint32_t)cb, (cuuint32_t)wp, (cuuint32_t)rows, 1};
@@ -238,6 +283,7 @@ static int encode_window(CUtensorMap *map, const void *ptr, int n, int h, int w,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(cb), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return set_error(SPARQ_ERR_CUDA, "cuTensorMapEncodeTiled (window) failed with CUresult %d", (int)r);
+    map_store(key, *map);
     return SPARQ_OK;
 }
 
@@ -248,13 +294,17 @@ static CUresult encode_weight_blocks(CUtensorMap *map, const void *ptr, int64_t 
 {
     static EncodeTiledFn fn = nullptr;
     if (!fn && driver_fn("cuTensorMapEncodeTiled", (void **)&fn) != SPARQ_OK) return CUDA_ERROR_NOT_FOUND;
+    const MapKey key = {{4, (uint64_t)(uintptr_t)ptr, (uint64_t)K, (uint64_t)cout, (uint64_t)cb, (uint64_t)bn, (uint64_t)blocks}};
+    if (map_lookup(key, map)) return CUDA_SUCCESS;
     cuuint64_t dims[3] = {(cuuint64_t)cb, (cuuint64_t)cout, (cuuint64_t)blocks};
     cuuint64_t strides[2] = {(cuuint64_t)K, (cuuint64_t)cb};
     cuuint32_t box[3] = {(cuuint32_t)cb, (cuuint32_t)bn, (cuuint32_t)blocks};
     cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(cb), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(cb), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r == CUDA_SUCCESS) map_store(key, *map);
+    return r;
 }
 
 constexpr int kMaxDynSmem = kWindowMaxDynSmem;
