@@ -386,6 +386,7 @@ struct EpiView {
     bool small_acc;   // |acc| < 2^22 guaranteed
     bool vec_ok;      // rows allow 16/32-byte vector stores
     bool u8_wide;     // 256-bit stores allowed on u8_out
+    bool lean;        // only requantized bytes are wanted and whole 32-byte groups can be stored: see epi_chunk_u8
     int next_mode;    // SPARQ mode applied to the requantized bytes (producer-side transform)
     int next_rnd;
     XformDev next_xf;
@@ -411,6 +412,8 @@ __device__ __forceinline__ EpiView make_epi_view(const Args &g)
     e.small_acc = g.K * (255 * 128) < (1 << 22);
     e.vec_ok = (g.N % 32) == 0;
     e.u8_wide = (reinterpret_cast<uintptr_t>(g.u8_out) & 31u) == 0;
+    e.lean = e.u8_out && !g.acc_out && !g.f32_out && !g.residual && g.next_mode == SPARQ_MODE_NONE && !e.relu_op &&
+             e.vec_ok && e.u8_wide;
     e.next_mode = g.next_mode;
     e.next_rnd = g.next_rnd;
     e.next_xf = g.next_xf;
@@ -534,6 +537,77 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[NV], i
     }
 }
 
+// Two fp32 values in one 64-bit register and the packed arithmetic of sm_100: each instruction
+// performs the IEEE round-to-nearest operation on both halves, so a pair of columns costs one
+// issue slot where the scalar form costs two.
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t r, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+// The form every layer of a network uses -- requantized bytes only, no residual, full 32-column
+// groups -- as straight-line code with nothing decided per element and the fp32 steps done two
+// columns at a time: per accumulator an exact int -> float step, one fma, one multiply, the
+// clamp and the rounding add, then three byte permutes per four columns.  Same IEEE sequence
+// per element as epi_chunk.
+template <bool SMALL>
+__device__ __forceinline__ void epi_chunk_u8(const EpiView &e, uint32_t (&v)[32], int64_t row, int64_t col0, int ct,
+                                             const float *s_scale, const float *s_bias)
+{
+    const uint64_t inv2 = f2_pack(e.inv_out_scale, e.inv_out_scale);
+    const uint64_t magic2 = f2_pack(12582912.0f, 12582912.0f);
+    const uint64_t neg_magic2 = f2_pack(-12582912.0f, -12582912.0f);
+    uint32_t w[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const float4 sc = *reinterpret_cast<const float4 *>(&s_scale[ct + 4 * q]);
+        const float4 bi = *reinterpret_cast<const float4 *>(&s_bias[ct + 4 * q]);
+        uint32_t b[4];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int32_t a0 = (int32_t)v[4 * q + 2 * h], a1 = (int32_t)v[4 * q + 2 * h + 1];
+            // (float)acc: exact through the add-based form when |acc| < 2^22
+            const uint64_t t = SMALL ? f2_add(f2_pack(__int_as_float(a0 + 0x4B400000), __int_as_float(a1 + 0x4B400000)), neg_magic2)
+                                     : f2_pack(__int2float_rn(a0), __int2float_rn(a1));
+            const uint64_t y = f2_fma(t, h ? f2_pack(sc.z, sc.w) : f2_pack(sc.x, sc.y), h ? f2_pack(bi.z, bi.w) : f2_pack(bi.x, bi.y));
+            float z0, z1;
+            f2_unpack(f2_mul(y, inv2), z0, z1);
+            z0 = fminf(fmaxf(z0, 0.0f), 255.0f);
+            z1 = fminf(fmaxf(z1, 0.0f), 255.0f);
+            float r0, r1;
+            f2_unpack(f2_add(f2_pack(z0, z1), magic2), r0, r1);
+            b[2 * h] = __float_as_uint(r0);
+            b[2 * h + 1] = __float_as_uint(r1);
+        }
+        w[q] = pack4(b[0], b[1], b[2], b[3]);
+    }
+    st_global_v8(e.u8_out + row * e.N + col0, w);
+}
+
 // A warp's share of one accumulator: CW (16, 32, 64 or 128) columns starting at
 // tensor-memory address taddr0 (tile-local column cbase), for this thread's output row.
 // After the last load has landed in registers the warp hands the accumulator back by
@@ -567,7 +641,12 @@ __device__ __forceinline__ void epi_warp_columns(const EpiView &e, uint32_t tadd
             const int ct = cbase + ch * 32;              // column inside the tile
             const int64_t col0 = n0 + ct;
             if (!row_ok || col0 >= e.N) continue;
-            epi_chunk<32, false>(e, v, row, col0, ct, s_scale, s_bias);
+            if (e.lean && col0 + 32 <= e.N) {
+                if (e.small_acc) epi_chunk_u8<true>(e, v, row, col0, ct, s_scale, s_bias);
+                else epi_chunk_u8<false>(e, v, row, col0, ct, s_scale, s_bias);
+            } else {
+                epi_chunk<32, false>(e, v, row, col0, ct, s_scale, s_bias);
+            }
         }
     }
 }
