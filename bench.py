@@ -44,7 +44,7 @@ WGT_BYTES = COUT * R * S * C
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 INT8_OVER_BF16 = 2.0     # nominal dense ratio (4.5 POPS int8 vs 2.25 PFLOPS bf16)
-CONV_TRAFFIC_BYTES = 6550272 + 0   # ncu, per launch; set to None whenever the kernel changes
+CONV_TRAFFIC_BYTES = 6550272 + 4864   # ncu dram read + write bytes per launch; set to None whenever the kernel changes
 # transform kernel (bSPARQ, n=4, 5opt, +R) captured on 2^28 activations: 268,445,184 B read +
 # 214,811,392 B written (the rest of the output is still dirty in L2); scales with the count
 TRANSFORM_TRAFFIC_PER_2P28 = 268445184 + 214811392
@@ -137,6 +137,28 @@ def time_region(fn, steps, warmup, sync):
     e1.record()
     sync()
     return e0.elapsed_time(e1)      # ms
+
+
+def time_graph(fn, steps, warmup, sync):
+    """Device time of `steps` calls captured in one CUDA graph (ms): the calls are enqueued
+    by the graph, not by Python, whose ~15 us per call would otherwise hide any kernel
+    shorter than that.  One untimed replay first (it uploads the graph)."""
+    import torch
+    for i in range(warmup):
+        fn(i)
+    sync()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(steps):
+            fn(warmup + i)
+    graph.replay()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync()
+    e0.record()
+    graph.replay()
+    e1.record()
+    sync()
+    return e0.elapsed_time(e1)
 
 
 def transform_section(device, pk, n, steps, warmup):
@@ -296,7 +318,7 @@ def extras(device, pk, steps):
         def step(i, xs=xs, os_=os_, wt=wt, sc=sc, bi=bi, inv=inv, L=L):
             sparq.sparq_conv2d_nhwc_s8(xs[i % len(xs)], wt, (L.stride, L.stride), (L.pad, L.pad), p,
                                        scale=sc, bias=bi, relu=True, inv_out_scale=inv, u8_out=os_[i % len(xs)])
-        ms = time_region(step, steps, 3, sync) / steps
+        ms = time_graph(step, steps, 3, sync) / steps
         ops = L.ops(64)
         layers.append({"layer": f"{L.h}x{L.w}x{L.cin}->{L.cout} {L.r}x{L.s}/s{L.stride}", "count": L.count,
                        "ms": round(ms, 4), "tops": round(ops / ms / 1e9, 1)})
