@@ -34,6 +34,11 @@ constexpr int kBM = 128;                 // rows of an output tile = MMA M
 constexpr int kNumEpiWarps = 8;          // two per tensor-memory lane quarter; without a transform
                                          // (mode NONE) the transform warps are epilogue warps too
 constexpr int kNumXfWarps = 8;
+// The transform warps work as two teams that take stages (or window pieces) alternately: a
+// stage's chain of barrier read, shared-memory loads, arithmetic, stores and fence is mostly
+// latency, and one team's chain overlaps the other's.
+constexpr int kXfTeams = 2;
+constexpr int kXfTeamWarps = kNumXfWarps / kXfTeams;
 constexpr int kFirstEpiWarp = 2;
 constexpr int kFirstXfWarp = kFirstEpiWarp + kNumEpiWarps;
 constexpr int kGemmThreads = 32 * (kFirstXfWarp + kNumXfWarps);
@@ -707,7 +712,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         prefetch_tensormap(&map_b);
         for (int s = 0; s < S; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
-            mbar_init(smem_u32(&bar_xf[s]), kNumXfWarps);
+            mbar_init(smem_u32(&bar_xf[s]), kXfTeamWarps);
             mbar_init(smem_u32(&bar_empty[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -861,35 +866,41 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
     } else if (MODE != SPARQ_MODE_NONE) {
         // ================= transform =================
-        const int xt = threadIdx.x - kFirstXfWarp * 32;            // 0 .. 255 among the transform threads
-        constexpr int kXfThreads = kNumXfWarps * 32;
+        const int team = (warp - kFirstXfWarp) / kXfTeamWarps;
+        const int xt = threadIdx.x - (kFirstXfWarp + team * kXfTeamWarps) * 32;   // 0 .. 127 inside the team
+        constexpr int kXfThreads = kXfTeamWarps * 32;
         constexpr int kVecs = Cfg::kABytes / 16;
         constexpr int kPerThread = kVecs / kXfThreads;
-        static_assert(kVecs % kXfThreads == 0, "A stage must split evenly over the transform threads");
+        constexpr int kBatch = kPerThread < 4 ? kPerThread : 4;     // vectors in flight per thread
+        static_assert(kVecs % kXfThreads == 0 && kPerThread % kBatch == 0, "A stage must split evenly over a team");
         const XformDev xf = g.xf;
         uint32_t it = 0;
         long long xw = 0;
         const long long xt0 = SPARQ_PROF_NOW();
         for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < kb_count; ++kb, ++it) {
+                if ((int)(it & 1u) != team) continue;      // the other team's stage
                 const int s = it % S;
                 SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_full[s]), (it / S) & 1, abort_flag, g.status));
                 const uint32_t base = a_stage(s) + (uint32_t)xt * 16u;
-                uint4 v[kPerThread];
 #pragma unroll
-                for (int j = 0; j < kPerThread; ++j)
-                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                                 : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w)
-                                 : "r"(base + (uint32_t)(j * kXfThreads * 16)));
+                for (int j0 = 0; j0 < kPerThread; j0 += kBatch) {
+                    uint4 v[kBatch];
 #pragma unroll
-                for (int j = 0; j < kPerThread; ++j) {
-                    v[j].x = xform_word<MODE, XN, RND, XN == 0>(v[j].x, xf);
-                    v[j].y = xform_word<MODE, XN, RND, XN == 0>(v[j].y, xf);
-                    v[j].z = xform_word<MODE, XN, RND, XN == 0>(v[j].z, xf);
-                    v[j].w = xform_word<MODE, XN, RND, XN == 0>(v[j].w, xf);
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
-                                 :: "r"(base + (uint32_t)(j * kXfThreads * 16)),
-                                    "r"(v[j].x), "r"(v[j].y), "r"(v[j].z), "r"(v[j].w) : "memory");
+                    for (int j = 0; j < kBatch; ++j)
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                     : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w)
+                                     : "r"(base + (uint32_t)((j0 + j) * kXfThreads * 16)));
+#pragma unroll
+                    for (int j = 0; j < kBatch; ++j) {
+                        v[j].x = xform_word<MODE, XN, RND, XN == 0>(v[j].x, xf);
+                        v[j].y = xform_word<MODE, XN, RND, XN == 0>(v[j].y, xf);
+                        v[j].z = xform_word<MODE, XN, RND, XN == 0>(v[j].z, xf);
+                        v[j].w = xform_word<MODE, XN, RND, XN == 0>(v[j].w, xf);
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
+                                     :: "r"(base + (uint32_t)((j0 + j) * kXfThreads * 16)),
+                                        "r"(v[j].x), "r"(v[j].y), "r"(v[j].z), "r"(v[j].w) : "memory");
+                    }
                 }
                 fence_proxy_async_smem();       // generic-proxy writes visible to the tensor core
                 __syncwarp();
