@@ -48,7 +48,7 @@ struct WindowArgs {
     int plane_bytes;        // shared-memory bytes reserved per channel block (>= rows the MMA may touch)
     int win_bufs;           // window buffers in the ring
     int b_stages;           // weight stages (stream mode) or resident blocks (resident mode)
-    int issuers;            // 1: warp 1 issues every tile; 2: the two issuer warps alternate
+    int issuers;            // 2: the two issuer warps alternate (resident weights); 1: warp 1 issues every tile (streamed weights)
     int w_one_copy;         // resident weights: map_w is the 3-D (bytes, rows, blocks) view and one copy brings all blocks
     uint32_t n_tiles;       // column tiles
     uint32_t units;         // n_img * tiles_per_img * n_tiles, column tile fastest

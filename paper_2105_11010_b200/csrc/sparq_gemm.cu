@@ -405,10 +405,10 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     WindowArgs g;
     memset(&g, 0, sizeof(g));
     g.w_one_copy = w_one_copy ? 1 : 0;
-    g.issuers = 2;
-#if defined(SPARQ_PROF) || defined(SPARQ_TUNE)
-    if (const char *ev = getenv("SPARQ_ISSUERS")) g.issuers = atoi(ev) == 1 ? 1 : 2;
-#endif
+    // Streamed weights pass through a ring that is shorter than one tile's blocks, in tile order:
+    // two issuers on different tiles would wait on the same stage barriers several phases apart,
+    // which a parity wait cannot tell apart.  One issuer then; two with resident weights.
+    g.issuers = resident ? 2 : 1;
     g.N = cout; g.K = K;
     g.n_img = n; g.H = h; g.W = w; g.C = c; g.R = r; g.S = s; g.pad_h = pad_h; g.pad_w = pad_w; g.Ho = ho; g.Wo = wo;
     g.Wp = wp; g.TR = tr; g.tiles_per_img = tiles_per_img; g.c_blocks = c_blocks;

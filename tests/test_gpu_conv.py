@@ -87,6 +87,23 @@ def test_stride1_filter_shapes_exact(cfg):
         check_full(x, wt, stride, pad, variant, seed=sum(cfg))
 
 
+@pytest.mark.parametrize("cfg", [
+    # more tiles than SMs, so that a CTA's share of the tile sequence holds several tiles: groups
+    # of tiles sharing one window, shares that cross image boundaries, short last groups
+    (12, 56, 56, 64, 64, 3, 3, 1, 1),     # 336 tiles of two rows: groups of three, 64-channel resident weights
+    (40, 28, 28, 128, 128, 3, 3, 1, 1),   # 280 tiles of four rows: groups of two beside 144 KB of weights
+    (30, 27, 28, 128, 128, 3, 3, 1, 1),   # last tile of every image has three rows
+    (80, 14, 14, 256, 256, 3, 3, 1, 1),   # two channel blocks, streamed weights, 256-wide tiles
+    (23, 28, 28, 128, 256, 3, 3, 1, 1),   # 161 tiles, two column tiles or one 256-wide
+])
+@pytest.mark.parametrize("variant", [V5, (sparq.MODE_NONE, 4, 0x1F, 1)])
+def test_grouped_windows_exact(cfg, variant):
+    nb, h, w, c, cout, r, s, stride, pad = cfg
+    x = synth.activations(sum(cfg) + 2, (nb, h, w, c), 0.45)
+    wt = synth.weights(sum(cfg) + 2, (cout, r, s, c))
+    check_full(x, wt, stride, pad, variant, seed=sum(cfg))
+
+
 def test_config2_resnet18_conv_full():
     # 32 x 56 x 56 x 64, 45% zeros, 3x3 stride 1 pad 1, 64 filters; scale, bias, ReLU, requant
     x = synth.activations(1, (32, 56, 56, 64), 0.45)
