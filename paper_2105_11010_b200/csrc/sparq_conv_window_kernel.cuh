@@ -499,6 +499,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 rs[i] = s_scale[cbase + i];
                 rb[i] = s_bias[cbase + i];
             }
+            uint32_t pre_full = 0;     // the next tile's accumulator was seen complete
             while (walk.next()) {
               for (int j = 0; j < (int)walk.cnt; ++j, ++wt) {
                 const uint32_t acc = wt & (uint32_t)(kAcc - 1);
@@ -507,13 +508,20 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 const bool row_ok = slot_ok && (oh < g.Ho);
                 uint8_t *dst = g.u8_out + (((int64_t)walk.img * g.Ho + oh) * g.Wo + ow) * 64 + cbase;
                 const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + (uint32_t)cbase;
-                SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status));
+                if (!pre_full) SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status));
                 tc_fence_after();
                 if (warp == kFirstEpiWarp && lane == 0) SPARQ_PROF_TL(1, 2 * wt, cta_t0);
+                pre_full = 0;
 #pragma unroll
                 for (int hh = 0; hh < kColsPerWarp / 16; ++hh) {
                     uint32_t v[16];
                     tmem_ld_32x16_issue(taddr0 + (uint32_t)(hh * 16), v);
+                    // While the load is in flight: has the next tile of the group been accumulated
+                    // already?  A barrier read takes hundreds of cycles behind the tensor core's
+                    // shared-memory traffic; here it overlaps the tensor-memory load, and a "yes"
+                    // lets the next tile start without one.
+                    if (hh == 0 && j + 1 < (int)walk.cnt)
+                        pre_full = mbar_test(smem_u32(&bar_acc_full[(wt + 1u) & (uint32_t)(kAcc - 1)]), ((wt + 1u) / (uint32_t)kAcc) & 1u);
                     tmem_ld_wait();
                     if (hh + 1 == kColsPerWarp / 16) {
                         tc_fence_before();

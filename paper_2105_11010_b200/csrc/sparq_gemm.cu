@@ -258,6 +258,7 @@ static int gemm_impl(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     rc = fill_common(&g, x, e, status);
     if (rc != SPARQ_OK) return rc;
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
+    if (tiles >= ((int64_t)1 << 31)) return set_error(SPARQ_ERR_UNSUPPORTED, "more than 2^31 output tiles");
     const int grid = (int)(tiles < sms ? tiles : sms);
     cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
     if (ce != cudaSuccess) return cuda_error(ce, "sparq_gemm_kernel launch");
@@ -460,6 +461,7 @@ int gemm_with_status(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     rc = fill_common(&g, x, e, status);
     if (rc != SPARQ_OK) return rc;
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
+    if (tiles >= ((int64_t)1 << 31)) return set_error(SPARQ_ERR_UNSUPPORTED, "more than 2^31 output tiles");
     const int grid = (int)(tiles < sms ? tiles : sms);
     cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
     if (ce != cudaSuccess) return cuda_error(ce, "sparq_gemm_kernel launch");
@@ -553,6 +555,7 @@ extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, in
     rc = fill_common(&g, x, e, status);
     if (rc != SPARQ_OK) return rc;
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((cout + bn - 1) / bn);
+    if (tiles >= ((int64_t)1 << 31)) return set_error(SPARQ_ERR_UNSUPPORTED, "more than 2^31 output tiles");
     const int grid = (int)(tiles < sms ? tiles : sms);
     cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
     if (ce != cudaSuccess) return cuda_error(ce, "sparq_gemm_kernel (convolution) launch");

@@ -737,7 +737,10 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
     const int64_t m_tiles = (g.M + kBM - 1) / kBM;
     const int64_t n_tiles = (g.N + BN - 1) / BN;
-    const int64_t total_tiles = m_tiles * n_tiles;
+    // tile indices fit 32 bits (the host refuses larger problems); a 64-bit division per tile
+    // and thread costs more instructions than a tile's share of the epilogue arithmetic
+    const uint32_t total_tiles = (uint32_t)(m_tiles * n_tiles);
+    const uint32_t n_tiles32 = (uint32_t)n_tiles;
     const int kb_count = g.k_blocks;
 
     if (warp == 0) {
@@ -746,15 +749,15 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             uint32_t it = 0;   // running stage counter across tiles
             long long pw = 0;
             const long long pt0 = SPARQ_PROF_NOW();
-            for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-                const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
-                const int64_t m0 = mt * kBM;
+            for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+                const uint32_t mt = (n_tiles32 == 1) ? tile : tile / n_tiles32, nt = tile - mt * n_tiles32;
+                const int64_t m0 = (int64_t)mt * kBM;
                 const int n0 = (int)(nt * BN);
                 int base_w = 0, base_h = 0, base_n = 0;
                 if (g.conv) {
-                    const int64_t hw = (int64_t)g.Ho * g.Wo;
-                    base_n = (int)(m0 / hw);
-                    const int rem = (int)(m0 % hw);
+                    const uint32_t hw = (uint32_t)(g.Ho * g.Wo), m032 = (uint32_t)m0;   // M of a convolution fits 31 bits
+                    base_n = (int)(m032 / hw);
+                    const int rem = (int)(m032 - (uint32_t)base_n * hw);
                     base_h = (rem / g.Wo) * g.stride_h - g.pad_h;
                     base_w = (rem % g.Wo) * g.stride_w - g.pad_w;
                 }
@@ -802,7 +805,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             uint32_t ph = 0;       // its phase parity
             long long mw = 0, ma = 0;
             const long long mt0 = SPARQ_PROF_NOW();
-            for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
+            for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
                 const int acc = local_tile & 1;
                 const uint32_t acc_use = local_tile >> 1;
                 if (acc_use > 0) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status));
@@ -843,8 +846,9 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         int64_t staged_nt = -1;
         long long ew = 0;
         const long long et0 = SPARQ_PROF_NOW();
-        for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
-            const int64_t mt = tile / n_tiles, nt = tile % n_tiles;
+        for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
+            const uint32_t mt32 = (n_tiles32 == 1) ? tile : tile / n_tiles32;
+            const int64_t mt = mt32, nt = tile - mt32 * n_tiles32;
             const int acc = local_tile & 1;
             const uint32_t acc_use = local_tile >> 1;
             if (ev.need_f && nt != staged_nt) {              // new column tile: new scale / bias
@@ -877,7 +881,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         uint32_t it = 0;
         long long xw = 0;
         const long long xt0 = SPARQ_PROF_NOW();
-        for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < kb_count; ++kb, ++it) {
                 if ((int)(it & 1u) != team) continue;      // the other team's stage
                 const int s = it % S;
