@@ -44,10 +44,13 @@ WGT_BYTES = COUT * R * S * C
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 INT8_OVER_BF16 = 2.0     # nominal dense ratio (4.5 POPS int8 vs 2.25 PFLOPS bf16)
-CONV_TRAFFIC_BYTES = 6550272 + 4864   # ncu dram read + write bytes per launch; set to None whenever the kernel changes
+CONV_TRAFFIC_BYTES = None   # ncu dram read + write bytes per launch; set to None whenever the kernel changes
 # transform kernel (bSPARQ, n=4, 5opt, +R) captured on 2^28 activations: 268,445,184 B read +
 # 214,811,392 B written (the rest of the output is still dirty in L2); scales with the count
 TRANSFORM_TRAFFIC_PER_2P28 = 268445184 + 214811392
+# fused GEMM kernel on the 56x56x64 -> 256 layer at batch 64: 12.92 MB read, 2.44 MB written per launch (most of
+# the 51 MB output is still dirty in L2 when the launch ends); None whenever that kernel changes
+LAYER1X1_TRAFFIC_BYTES = 12924672 + 2441216
 
 
 def peaks():
@@ -246,6 +249,44 @@ def frontend_section(device, pk, n, steps, warmup):
     return res
 
 
+def layer1x1_section(device, pk, steps, warmup):
+    """The fused GEMM kernel on an output-heavy 1x1 layer of the ResNet-50 stack at batch 64
+    (56x56x64 -> 256: M 200704, K 64, N 256; vSPARQ n = 4, five placements, round; scale + bias +
+    ReLU + requantize).  Bandwidth-side roofline: bytes = input + output + weights."""
+    import torch
+    import paper_2105_11010_b200 as sparq
+    sync = torch.cuda.synchronize
+    nb, hw, c, cout = 64, 56, 64, 256
+    sets = 4                                         # 4 x (12.8 MB in + 51.4 MB out) = 257 MB > L2
+    gen = torch.Generator(device=device).manual_seed(9)
+    xs = []
+    for _ in range(sets):
+        z = torch.randn(nb * hw * hw * c, generator=gen, device=device)
+        v = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
+        v[torch.rand(v.numel(), generator=gen, device=device) < 0.5] = 0
+        xs.append(v.view(nb, hw, hw, c))
+        del z
+    outs = [torch.empty((nb, hw, hw, cout), dtype=torch.uint8, device=device) for _ in range(sets)]
+    wt = torch.from_numpy(synth.weights(9, (cout, 1, 1, c))).to(device)
+    sc = torch.from_numpy(synth.scales(9, cout)).to(device)
+    bi = torch.from_numpy(synth.bias(9, cout)).to(device)
+    inv = synth.inv_out_scale(c, 0.5)
+    p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+
+    def step(i):
+        sparq.sparq_conv2d_nhwc_s8(xs[i % sets], wt, (1, 1), (0, 0), p, scale=sc, bias=bi, relu=True,
+                                   inv_out_scale=inv, u8_out=outs[i % sets])
+    ms = time_graph(step, steps, warmup, sync) / steps
+    sparq.sparq_check()
+    nbytes = nb * hw * hw * (c + cout) + cout * c
+    gbs = nbytes / ms / 1e6
+    return {"layer": "56x56x64->256 1x1/s1, batch 64", "ms": round(ms, 4),
+            "tops": round(2 * nb * hw * hw * c * cout / ms / 1e9, 1), "gbs": round(gbs, 1),
+            "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
+                         "frac": round(gbs / pk["hbm"], 4), "traffic": LAYER1X1_TRAFFIC_BYTES, "peak_source": pk["source"] + " copy",
+                         "kernel": "sparq_gemm_kernel<256,64,VSPARQ,4,round>", "algorithmic_bytes_per_launch": nbytes}}
+
+
 def sparse24_section(device, pk, steps, warmup):
     """vSPARQ on 2:4 sparse weights, shape of the 28x28x128 -> 128 3x3 layer at batch 128
     (M 100352, K 1152, N 128): expansion of the activations (bytes = M*K read + 3*M*K
@@ -294,6 +335,7 @@ def extras(device, pk, steps):
     out["packed_stream_2p28"] = pack_section(device, pk, 1 << 28, 20, 3)
     out["minmax_frontend_2p28"] = frontend_section(device, pk, 1 << 28, 20, 3)
     out["sparse24_vsparq"] = sparse24_section(device, pk, 20, 3)
+    out["gemm_layer1x1"] = layer1x1_section(device, pk, 20, 3)
     # --- ResNet-50 sweep, batch 64, every conv shape (22 shapes, 52 instances) ---
     p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
     layers, total_ms, total_ops = [], 0.0, 0
@@ -401,7 +443,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the transform and ResNet-50 sweep sections")
-    ap.add_argument("--section", default="main", choices=["main", "transform", "pack", "frontend", "sparse24"],
+    ap.add_argument("--section", default="main", choices=["main", "transform", "pack", "frontend", "sparse24", "layer1x1"],
                     help="'transform' times only the standalone transform kernel (small, for profiling)")
     ap.add_argument("--log2n", type=int, default=28, help="activations for --section transform (2^log2n)")
     args = ap.parse_args()
@@ -445,6 +487,9 @@ def main():
         return
     if args.section == "pack":
         print(json.dumps(pack_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
+        return
+    if args.section == "layer1x1":
+        print(json.dumps(layer1x1_section(device, pk, args.steps, args.warmup)))
         return
     sets = 20   # 20 x (6.4 MB in + 6.4 MB out) = 257 MB > 126 MB of L2
     xs, outs, wt, scale, bias = build_layer(device, sets)

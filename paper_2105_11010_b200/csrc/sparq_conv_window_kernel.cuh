@@ -179,7 +179,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
         // barrier set-up spread over the lanes of one warp
         for (int b = lane; b < kMaxWinBufs * kMaxG; b += 32) {
             mbar_init(smem_u32(&bar_win_full[b]), 1);
-            mbar_init(smem_u32(&bar_win_xf[b]), kXfTeamWarps);    // the team that owns the piece
+            mbar_init(smem_u32(&bar_win_xf[b]), kNumXfWarps);
         }
         if (lane < kMaxWinBufs) mbar_init(smem_u32(&bar_win_empty[lane]), 2);     // one arrival per issuing warp
         if (lane < kMaxBStages) {
@@ -358,13 +358,13 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 0, cta_t0);
                     if (acc_use > 0 && !pre_acc) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status));
                     if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 1, cta_t0);
-                    // Tile j reads pieces 0..j.  Neither the copies nor the two transform teams
-                    // (which take pieces alternately) finish pieces in order, so this issuer waits
-                    // for pieces j-1 and j; its previous tile of the group, j-2, waited for the two
-                    // before.
+                    // Tile j reads pieces 0..j.  The transform warps finish pieces in order, so with
+                    // a transform piece j's barrier covers the earlier ones.  Without one the copies
+                    // land in any order: this issuer waits for pieces j-1 and j (its previous tile
+                    // of the group, j-2, waited for the two before).
                     const uint32_t ops_bar = smem_u32(MODE == SPARQ_MODE_NONE ? &bar_win_full[b * kMaxG + j] : &bar_win_xf[b * kMaxG + j]);
                     if (!pre_ops) {
-                        if (j > 0) SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar - 8u, wph, abort_flag, g.status));
+                        if (MODE == SPARQ_MODE_NONE && j > 0) SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar - 8u, wph, abort_flag, g.status));
                         SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar, wph, abort_flag, g.status));
                     }
                     tc_fence_after();
@@ -378,7 +378,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                         const uint32_t m = mbar_test3(nuse ? smem_u32(&bar_acc_empty[nacc]) : ops_bar, nuse ? (nuse - 1u) & 1u : wph,
                                                       ops_bar + 8u, wph, ops_bar + 8u * step, wph);
                         pre_acc = nuse ? (m & 1u) : 1u;
-                        pre_ops = (uint32_t)((m & 6u) == 6u);
+                        pre_ops = (MODE == SPARQ_MODE_NONE) ? (uint32_t)((m & 6u) == 6u) : (m >> 2);
                     };
                     const uint64_t a_desc0 = a_grp + (uint64_t)((uint32_t)j * tile16);
                     const long long is0 = SPARQ_PROF_NOW();
@@ -437,13 +437,11 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 }
                 // The buffer goes back to the producer once both issuers have arrived and their
                 // MMAs have retired.  With a transform, first make sure that every transform warp
-                // is past all of this use's barriers (each team arrives on its last piece's barrier
-                // last, and those are the buffer's last two), so that none of them can still be
-                // waiting on a phase when the producer starts the next.
-                if (MODE != SPARQ_MODE_NONE && (int)walk.cnt < g.G) {
+                // is past all of this use's barriers (they arrive on the last piece's barrier
+                // last), so that none of them can still be waiting on a phase when the producer
+                // starts the next.
+                if (MODE != SPARQ_MODE_NONE && (int)walk.cnt < g.G)
                     SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b * kMaxG + g.G - 1]), wph, abort_flag, g.status));
-                    SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b * kMaxG + g.G - 2]), wph, abort_flag, g.status));
-                }
                 if (issued) {
                     tc_commit_if(smem_u32(&bar_win_empty[b]), elected);
                 } else {
@@ -575,10 +573,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
         }
     } else if (MODE != SPARQ_MODE_NONE) {
         // ================= transform: once per piece =================
-        // two teams; team t rewrites the pieces with index parity t
-        const uint32_t team = (uint32_t)(warp - kFirstXfWarp) / kXfTeamWarps;
-        const uint32_t xt = threadIdx.x - (kFirstXfWarp + team * kXfTeamWarps) * 32;
-        constexpr uint32_t kXfThreads = kXfTeamWarps * 32;
+        const uint32_t xt = threadIdx.x - kFirstXfWarp * 32;
+        constexpr uint32_t kXfThreads = kNumXfWarps * 32;
         const XformDev xf = g.xf;
         uint32_t gi = 0;
         long long xw = 0;
@@ -586,7 +582,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
         while (walk.next()) {
             const int b = gi % g.win_bufs;
             const uint32_t wph = (gi / g.win_bufs) & 1u;
-            for (int j = (int)team; j < g.G; j += kXfTeams) {
+            for (int j = 0; j < g.G; ++j) {
                 SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), wph, abort_flag, g.status));
                 if (warp == kFirstXfWarp && lane == 0 && gi == 0) SPARQ_PROF_TL(2, 2 * j, cta_t0);
                 if (j < (int)walk.cnt) {
