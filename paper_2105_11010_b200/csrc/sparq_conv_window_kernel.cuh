@@ -205,23 +205,26 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    // this CTA's share of the tile sequence: kernel arguments only, so it is worked out (two
+    // integer divisions) while the previous kernel may still be running
+    GroupWalk walk(g);
     dep_launch();
     dep_wait();
 
-    GroupWalk walk(g);
     if (threadIdx.x == 0) SPARQ_PROF_STORE(15, SPARQ_PROF_NOW() - cta_t0);
 
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            uint32_t gi = 0;      // group counter
+            uint32_t gi = 0;                   // group counter
+            int rb = 0; uint32_t ruse = 0;     // its window buffer (gi % win_bufs) and that buffer's use count (gi / win_bufs)
             uint32_t it = 0;      // streamed weight-block counter
             bool b_issued = false;  // resident weights requested
             long long pw = 0;
             const long long pt0 = SPARQ_PROF_NOW();
             while (walk.next()) {
-                const int b = gi % g.win_bufs;
-                const uint32_t use = gi / g.win_bufs;
+                const int b = rb;                 // window buffer of this group and how often it was used before
+                const uint32_t use = ruse;
                 if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_win_empty[b]), (use - 1) & 1, abort_flag, g.status));
                 if (*abort_flag) break;
                 const int oh0 = (int)walk.tin * g.TR;
@@ -267,6 +270,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 }
 #endif
                 ++gi;
+                if (++rb == g.win_bufs) { rb = 0; ++ruse; }
                 if (!B_RESIDENT) {
                     bool stop = false;
                     for (int j = 0; j < (int)walk.cnt && !stop; ++j) {
@@ -320,7 +324,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             const uint64_t win_desc0 = make_smem_desc<CB>(smem_base);
             const uint64_t b_desc0 = make_smem_desc<CB>(b_base);
             uint32_t wt = 0;                   // tile counter (both issuers count every tile)
-            uint32_t gi = 0;                   // group counter (window buffer and phase)
+            uint32_t gi = 0;                   // group counter
+            int rb = 0; uint32_t ruse = 0;     // its window buffer (gi % win_bufs) and that buffer's use count (gi / win_bufs)
             int s = 0;  uint32_t bph = 0;      // streamed weight stage and its phase parity
             long long mw = 0, ma = 0, mb = 0, mi = 0;
             const long long mt0 = SPARQ_PROF_NOW();
@@ -331,8 +336,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             const uint32_t tile16 = (uint32_t)(g.TR * g.Wp * CB) >> 4;
             if (B_RESIDENT) SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status));
             while (walk.next()) {
-                const int b = gi % g.win_bufs;
-                const uint32_t wph = (gi / g.win_bufs) & 1u;
+                const int b = rb;
+                const uint32_t wph = ruse & 1u;
                 const uint64_t a_grp = win_desc0 + (uint64_t)((uint32_t)b * (win_bytes >> 4));
                 bool issued = false;
                 // Barrier reads go through the shared-memory pipe, which the tensor core's operand
@@ -452,6 +457,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     if (elected) mbar_arrive(smem_u32(&bar_win_empty[b]));
                 }
                 ++gi;
+                if (++rb == g.win_bufs) { rb = 0; ++ruse; }
             }
             if (me == 0) {
                 SPARQ_PROF_STORE(2, mw);
@@ -577,11 +583,12 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
         constexpr uint32_t kXfThreads = kNumXfWarps * 32;
         const XformDev xf = g.xf;
         uint32_t gi = 0;
+        int rb = 0; uint32_t ruse = 0;         // window buffer of the group (gi % win_bufs) and its use count (gi / win_bufs)
         long long xw = 0;
         const long long xt0 = SPARQ_PROF_NOW();
         while (walk.next()) {
-            const int b = gi % g.win_bufs;
-            const uint32_t wph = (gi / g.win_bufs) & 1u;
+            const int b = rb;
+            const uint32_t wph = ruse & 1u;
             for (int j = 0; j < g.G; ++j) {
                 SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), wph, abort_flag, g.status));
                 if (warp == kFirstXfWarp && lane == 0 && gi == 0) SPARQ_PROF_TL(2, 2 * j, cta_t0);
@@ -622,6 +629,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 if (warp == kFirstXfWarp && lane == 0 && gi == 0) SPARQ_PROF_TL(2, 2 * j + 1, cta_t0);
             }
             ++gi;
+                if (++rb == g.win_bufs) { rb = 0; ++ruse; }
         }
         if (warp == kFirstXfWarp && lane == 0) {
             SPARQ_PROF_STORE(7, xw);
