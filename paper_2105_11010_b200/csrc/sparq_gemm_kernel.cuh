@@ -47,7 +47,7 @@ __host__ __device__ constexpr int epi_warps(int mode) { return mode == SPARQ_MOD
 constexpr int kSmemBudget = 200 * 1024;  // for the stage ring
 constexpr long long kWaitLimitCycles = 2000000000LL;
 
-// Optional per-role cycle counters (builds with -DSPARQ_PROF only): how long each warp role
+// Optional per-role cycle counters (builds with -DSPARQ_PROF -rdc=true only): how long each warp role
 // waited on its barriers and how long it ran, per CTA.  Compiled out otherwise.
 #ifdef SPARQ_PROF
 extern __device__ long long g_prof[148 * 16];

@@ -133,3 +133,26 @@ def test_rejected_arguments():
     with pytest.raises(sparq.SparqError):
         sparq.sparq_gemm_s8(A, B, sparq.SparqParams(), u8_out=torch.zeros((128, 64), dtype=torch.uint8, device="cuda"))  # no scale
     sparq.sparq_gemm_s8(A[:0], B, sparq.SparqParams(), acc_out=acc)        # M == 0: no-op
+
+
+@pytest.mark.parametrize("shape", [
+    # M, K, N: the requantized-bytes-only form takes its own straight-line epilogue path
+    (1000, 64, 256),      # short reduction (add-based int -> float), ragged last row tile
+    (777, 128, 96),       # last column group of a warp only partly inside N: general path for it
+    (2048, 576, 64),      # long reduction (conversion-based int -> float), 64-wide tiles
+    (300, 1024, 512),     # two column tiles of 256
+    (20000, 64, 128),     # more tiles than SMs
+])
+@pytest.mark.parametrize("mode", [sparq.MODE_VSPARQ, sparq.MODE_NONE])
+@pytest.mark.parametrize("relu", [True, False])
+def test_bytes_only_output_exact(shape, mode, relu):
+    M, K, N = shape
+    seed = 7000 + M + K + N
+    A = synth.activations(seed, (M, K), 0.5)
+    B = synth.weights(seed + 1, (K, N))
+    scale, bias = synth.scales(seed + 2, N), synth.bias(seed + 3, N)
+    inv = synth.inv_out_scale(K)
+    got = gpu_gemm(A, B, sparq.SparqParams(mode, 4, 0x1F, 1), scale, bias, relu, inv, want=("u8",))
+    acc = oracle.gemm(A, B, mode, 4, 0x1F, 1)
+    _, q = oracle.epilogue(acc, scale, bias, relu, inv)
+    assert np.array_equal(got["u8"], q)
