@@ -169,7 +169,17 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
 
     const int taps = g.R * g.S;
     const int kb_count = taps * g.c_blocks;            // weight blocks per tile
-
+    // A tile's epilogue is mostly latency (barrier read, tensor-memory loads, stores), not
+    // arithmetic.  When only requantized bytes are wanted and there is one column tile, the epilogue
+    // warps split into two teams, one per accumulator stage, each warp taking twice the columns of
+    // its lane quarter, so that the epilogues of two consecutive tiles overlap.
+    // (Measured: a gain on 64-wide tiles and on 128-wide tiles with a transform, whose eight epilogue
+    // warps are latency-bound; a loss where sixteen warps are already bound by instruction issue or
+    // where a warp would hold a 256-column accumulator for eight loads.)
+    constexpr bool kTeamsPay = BN == 64 || (BN == 128 && MODE != SPARQ_MODE_NONE);
+    const bool epi_teams = kTeamsPay && g.u8_out && !g.acc_out && !g.f32_out && !g.residual && g.next_mode == SPARQ_MODE_NONE &&
+                           g.n_tiles == 1 && (g.N % 32) == 0 && (!g.relu || g.inv_out_scale > 0.0f) &&
+                           (reinterpret_cast<uintptr_t>(g.u8_out) & 31u) == 0;
     if (threadIdx.x == 0) {
         prefetch_tensormap(&map_x0);
         prefetch_tensormap(&map_x1);
@@ -188,7 +198,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
         }
         if (lane < kAcc) {
             mbar_init(smem_u32(&bar_acc_full[lane]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[lane]), epi_warps(MODE));
+            mbar_init(smem_u32(&bar_acc_empty[lane]), epi_teams ? epi_warps(MODE) / 2 : epi_warps(MODE));
         }
         if (lane == 0) {
             mbar_init(smem_u32(&bar_done), 2);
@@ -494,6 +504,39 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
         // the scale and bias of its columns in registers for the whole launch -- shared-memory
         // reads queue behind the tensor core's operand fetches -- and takes the accumulator in
         // 16-column pieces so that those registers fit beside it.
+        if (epi_teams) {
+            constexpr int kTeamWarps = kEpi / 2;
+            constexpr int kTeamCols = BN / (kTeamWarps / 4);      // columns per warp
+            epi_stage_scale_bias<kEpi>(g, 0, BN, et, s_scale, s_bias);
+            const uint32_t team = (uint32_t)(warp - kFirstEpiWarp) / kTeamWarps;     // kAcc == 2: team t owns stage t
+            const int cbase = (((warp - kFirstEpiWarp) % kTeamWarps) >> 2) * kTeamCols;
+            while (walk.next()) {
+                for (int j = 0; j < (int)walk.cnt; ++j, ++wt) {
+                    if ((wt & 1u) != team) continue;
+                    const int oh = ((int)walk.tin + j) * g.TR + tr;
+                    const bool row_ok = slot_ok && (oh < g.Ho);
+                    const int64_t row = ((int64_t)walk.img * g.Ho + oh) * g.Wo + ow;
+                    const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + team * BN + (uint32_t)cbase;
+                    SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[team]), (wt >> 1) & 1u, abort_flag, g.status));
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int ch = 0; ch < kTeamCols / 32; ++ch) {
+                        uint32_t v[32];
+                        tmem_ld_32x32_issue(taddr0 + (uint32_t)(ch * 32), v);
+                        tmem_ld_wait();
+                        if (ch + 1 == kTeamCols / 32) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[team]));
+                        }
+                        const int ct = cbase + ch * 32;
+                        if (!row_ok || ct >= (int)g.N) continue;       // N is a multiple of 32 here
+                        if (ev.small_acc) epi_chunk_u8<true>(ev, v, row, ct, ct, s_scale, s_bias);
+                        else epi_chunk_u8<false>(ev, v, row, ct, ct, s_scale, s_bias);
+                    }
+                }
+            }
+        } else
         if (BN == 64 && ev.need_f && !g.acc_out && !g.f32_out && !g.residual && g.N == 64) {
             epi_stage_scale_bias<kEpi>(g, 0, BN, et, s_scale, s_bias);
             const int cbase = part * kColsPerWarp;
