@@ -508,7 +508,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             constexpr int kTeamWarps = kEpi / 2;
             constexpr int kTeamCols = BN / (kTeamWarps / 4);      // columns per warp
             epi_stage_scale_bias<kEpi>(g, 0, BN, et, s_scale, s_bias);
-            const uint32_t team = (uint32_t)(warp - kFirstEpiWarp) / kTeamWarps;     // kAcc == 2: team t owns stage t
+            const uint32_t team = (uint32_t)(warp - kFirstEpiWarp) / kTeamWarps;     // team t takes the tiles of parity t (kAcc is even)
             const int cbase = (((warp - kFirstEpiWarp) % kTeamWarps) >> 2) * kTeamCols;
             while (walk.next()) {
                 for (int j = 0; j < (int)walk.cnt; ++j, ++wt) {
@@ -516,8 +516,9 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     const int oh = ((int)walk.tin + j) * g.TR + tr;
                     const bool row_ok = slot_ok && (oh < g.Ho);
                     const int64_t row = ((int64_t)walk.img * g.Ho + oh) * g.Wo + ow;
-                    const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + team * BN + (uint32_t)cbase;
-                    SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[team]), (wt >> 1) & 1u, abort_flag, g.status));
+                    const uint32_t acc = wt & (uint32_t)(kAcc - 1);
+                    const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + (uint32_t)cbase;
+                    SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status));
                     tc_fence_after();
 #pragma unroll 1
                     for (int ch = 0; ch < kTeamCols / 32; ++ch) {
@@ -527,7 +528,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                         if (ch + 1 == kTeamCols / 32) {
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[team]));
+                            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
                         }
                         const int ct = cbase + ch * 32;
                         if (!row_ok || ct >= (int)g.N) continue;       // N is a multiple of 32 here
