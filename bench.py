@@ -44,7 +44,7 @@ WGT_BYTES = COUT * R * S * C
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 INT8_OVER_BF16 = 2.0     # nominal dense ratio (4.5 POPS int8 vs 2.25 PFLOPS bf16)
-CONV_TRAFFIC_BYTES = None   # ncu dram read + write bytes per launch; set to None whenever the kernel changes
+CONV_TRAFFIC_BYTES = 6541824 + 0   # ncu dram read + write bytes per launch; set to None whenever the kernel changes
 # transform kernel (bSPARQ, n=4, 5opt, +R) captured on 2^28 activations: 268,445,184 B read +
 # 214,811,392 B written (the rest of the output is still dirty in L2); scales with the count
 TRANSFORM_TRAFFIC_PER_2P28 = 268445184 + 214811392
