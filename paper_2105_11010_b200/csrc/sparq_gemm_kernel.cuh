@@ -707,6 +707,13 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     auto a_stage = [&](int s) { return smem_base + (uint32_t)s * Cfg::kStageBytes; };
     auto b_stage = [&](int s) { return smem_base + (uint32_t)s * Cfg::kStageBytes + Cfg::kABytes; };
 
+    // A tile's epilogue is mostly latency (barrier read, tensor-memory loads, stores).  On 64-wide
+    // tiles, and on 128-wide tiles with a transform (eight epilogue warps), with one column tile and
+    // only requantized bytes wanted, the epilogue warps split into two teams, one per accumulator
+    // stage, each warp taking twice the columns of its lane quarter: two tiles' epilogues overlap.
+    constexpr bool kTeamsPay = BN == 64 || (BN == 128 && MODE != SPARQ_MODE_NONE);
+    const bool epi_teams = kTeamsPay && g.N <= BN && make_epi_view(g).lean;
+
     if (threadIdx.x == 0) {
         prefetch_tensormap(&map_a);
         prefetch_tensormap(&map_b);
@@ -717,7 +724,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&bar_acc_full[a]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[a]), epi_warps(MODE));
+            mbar_init(smem_u32(&bar_acc_empty[a]), epi_teams ? epi_warps(MODE) / 2 : epi_warps(MODE));
         }
         mbar_init(smem_u32(&bar_done), 1);
         abort_word = 0;
@@ -846,6 +853,36 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         int64_t staged_nt = -1;
         long long ew = 0;
         const long long et0 = SPARQ_PROF_NOW();
+        if (epi_teams) {
+            constexpr int kTeamWarps = kEpi / 2;
+            constexpr int kTeamCols = BN / (kTeamWarps / 4);          // columns per warp
+            epi_stage_scale_bias<kEpi>(g, 0, BN, et, s_scale, s_bias);
+            const uint32_t team = (uint32_t)(warp - kFirstEpiWarp) / kTeamWarps;   // team t takes the tiles of parity t
+            const int tcbase = (((warp - kFirstEpiWarp) % kTeamWarps) >> 2) * kTeamCols;
+            for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
+                if ((local_tile & 1u) != team) continue;
+                const int64_t row = (int64_t)tile * kBM + quarter * 32 + lane;    // one column tile: row tile = tile
+                const bool row_ok = row < g.M;
+                const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + team * BN + (uint32_t)tcbase;
+                SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[team]), (local_tile >> 1) & 1u, abort_flag, g.status));
+                tc_fence_after();
+#pragma unroll 1
+                for (int ch = 0; ch < kTeamCols / 32; ++ch) {
+                    uint32_t v[32];
+                    tmem_ld_32x32_issue(taddr0 + (uint32_t)(ch * 32), v);
+                    tmem_ld_wait();
+                    if (ch + 1 == kTeamCols / 32) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[team]));
+                    }
+                    const int ct = tcbase + ch * 32;
+                    if (!row_ok || ct >= (int)g.N) continue;          // N is a multiple of 32 here
+                    if (ev.small_acc) epi_chunk_u8<true>(ev, v, row, ct, ct, s_scale, s_bias);
+                    else epi_chunk_u8<false>(ev, v, row, ct, ct, s_scale, s_bias);
+                }
+            }
+        } else
         for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
             const uint32_t mt32 = (n_tiles32 == 1) ? tile : tile / n_tiles32;
             const int64_t mt = mt32, nt = tile - mt32 * n_tiles32;
