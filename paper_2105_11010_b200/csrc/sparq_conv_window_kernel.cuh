@@ -63,6 +63,7 @@ struct WindowArgs {
     float *f32_out;
     uint8_t *u8_out;
     unsigned int *status;
+    long long wait_limit;   // cycles after which a device-side wait gives up
     // producer-side transform of u8_out (mode NONE = off)
     int next_mode, next_rnd;
     XformDev next_xf;
@@ -235,7 +236,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             while (walk.next()) {
                 const int b = rb;                 // window buffer of this group and how often it was used before
                 const uint32_t use = ruse;
-                if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_win_empty[b]), (use - 1) & 1, abort_flag, g.status));
+                if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_win_empty[b]), (use - 1) & 1, abort_flag, g.status, g.wait_limit));
                 if (*abort_flag) break;
                 const int oh0 = (int)walk.tin * g.TR;
                 if (gi == 0) SPARQ_PROF_STORE(9, SPARQ_PROF_NOW() - pt0);
@@ -274,7 +275,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 if (gi == 0) {
                     SPARQ_PROF_TL(3, 1, cta_t0);
                     for (int j = 0; j < (int)walk.cnt; ++j) {
-                        mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), 0, abort_flag, g.status);
+                        mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), 0, abort_flag, g.status, g.wait_limit);
                         SPARQ_PROF_TL(3, 2 + j, cta_t0);
                     }
                 }
@@ -288,7 +289,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                             for (int tap = 0; tap < taps; ++tap, ++it) {
                                 const int s = it % g.b_stages;
                                 const uint32_t buse = it / g.b_stages;
-                                if (buse > 0) mbar_wait(smem_u32(&bar_b_empty[s]), (buse - 1) & 1, abort_flag, g.status);
+                                if (buse > 0) mbar_wait(smem_u32(&bar_b_empty[s]), (buse - 1) & 1, abort_flag, g.status, g.wait_limit);
                                 if (*abort_flag) { stop = true; break; }
                                 const uint32_t full = smem_u32(&bar_b_full[s]);
                                 mbar_expect_tx(full, kBBlock);
@@ -307,13 +308,13 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 for (uint32_t q = gfirst; q < gi; ++q)
                     for (int j = 0; j < g.G; ++j)
                         mbar_wait(smem_u32(&bar_win_full[(q % g.win_bufs) * kMaxG + j]), (q / g.win_bufs) & 1,
-                                  abort_flag, g.status, true);
+                                  abort_flag, g.status, g.wait_limit, true);
                 if (B_RESIDENT) {
-                    if (b_issued) mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, true);
+                    if (b_issued) mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, g.wait_limit, true);
                 } else {
                     const uint32_t first = it > (uint32_t)g.b_stages ? it - g.b_stages : 0;
                     for (uint32_t q = first; q < it; ++q)
-                        mbar_wait(smem_u32(&bar_b_full[q % g.b_stages]), (q / g.b_stages) & 1, abort_flag, g.status, true);
+                        mbar_wait(smem_u32(&bar_b_full[q % g.b_stages]), (q / g.b_stages) & 1, abort_flag, g.status, g.wait_limit, true);
                 }
             }
         }
@@ -344,7 +345,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             const uint32_t row16 = (uint32_t)(g.Wp * CB) >> 4;
             const uint32_t plane16 = (uint32_t)g.plane_bytes >> 4;
             const uint32_t tile16 = (uint32_t)(g.TR * g.Wp * CB) >> 4;
-            if (B_RESIDENT) SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status));
+            if (B_RESIDENT) SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, g.wait_limit));
             while (walk.next()) {
                 const int b = rb;
                 const uint32_t wph = ruse & 1u;
@@ -371,7 +372,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     const uint32_t acc_use = wt / (uint32_t)kAcc;
                     const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
                     if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 0, cta_t0);
-                    if (acc_use > 0 && !pre_acc) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status));
+                    if (acc_use > 0 && !pre_acc) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status, g.wait_limit));
                     if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 1, cta_t0);
                     // Tile j reads pieces 0..j.  The transform warps finish pieces in order, so with
                     // a transform piece j's barrier covers the earlier ones.  Without one the copies
@@ -379,8 +380,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     // of the group, j-2, waited for the two before).
                     const uint32_t ops_bar = smem_u32(MODE == SPARQ_MODE_NONE ? &bar_win_full[b * kMaxG + j] : &bar_win_xf[b * kMaxG + j]);
                     if (!pre_ops) {
-                        if (MODE == SPARQ_MODE_NONE && j > 0) SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar - 8u, wph, abort_flag, g.status));
-                        SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar, wph, abort_flag, g.status));
+                        if (MODE == SPARQ_MODE_NONE && j > 0) SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar - 8u, wph, abort_flag, g.status, g.wait_limit));
+                        SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar, wph, abort_flag, g.status, g.wait_limit));
                     }
                     tc_fence_after();
                     pre_acc = pre_ops = 0;
@@ -407,7 +408,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                         if (B_RESIDENT) {
                             bdesc = b_desc0 + (uint64_t)(slot * (uint32_t)(kBBlock >> 4));
                         } else {
-                            SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status));
+                            SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status, g.wait_limit));
                             tc_fence_after();
                             bdesc = b_desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kBBlock >> 4));
                         }
@@ -456,14 +457,14 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 // last), so that none of them can still be waiting on a phase when the producer
                 // starts the next.
                 if (MODE != SPARQ_MODE_NONE && (int)walk.cnt < g.G)
-                    SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b * kMaxG + g.G - 1]), wph, abort_flag, g.status));
+                    SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b * kMaxG + g.G - 1]), wph, abort_flag, g.status, g.wait_limit));
                 if (issued) {
                     tc_commit_if(smem_u32(&bar_win_empty[b]), elected);
                 } else {
                     // No tile of this group was this issuer's.  It arrives only once the producer has
                     // started this use of the buffer (its first piece has landed), i.e. after the
                     // previous use's phase of the barrier has completed.
-                    mbar_wait(smem_u32(&bar_win_full[b * kMaxG]), wph, abort_flag, g.status);
+                    mbar_wait(smem_u32(&bar_win_full[b * kMaxG]), wph, abort_flag, g.status, g.wait_limit);
                     if (elected) mbar_arrive(smem_u32(&bar_win_empty[b]));
                 }
                 ++gi;
@@ -478,7 +479,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             }
             // all tensor-core work of this CTA has retired before tensor memory is freed
             tc_commit_if(smem_u32(&bar_done), elected);
-            mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, true);
+            mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, g.wait_limit, true);
             if (me == 0) SPARQ_PROF_TL(0, 40, cta_t0);
         }
         __syncwarp();
@@ -518,7 +519,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     const int64_t row = ((int64_t)walk.img * g.Ho + oh) * g.Wo + ow;
                     const uint32_t acc = wt & (uint32_t)(kAcc - 1);
                     const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + (uint32_t)cbase;
-                    SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status));
+                    SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status, g.wait_limit));
                     tc_fence_after();
 #pragma unroll 1
                     for (int ch = 0; ch < kTeamCols / 32; ++ch) {
@@ -556,7 +557,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 const bool row_ok = slot_ok && (oh < g.Ho);
                 uint8_t *dst = g.u8_out + (((int64_t)walk.img * g.Ho + oh) * g.Wo + ow) * 64 + cbase;
                 const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + (uint32_t)cbase;
-                if (!pre_full) SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status));
+                if (!pre_full) SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status, g.wait_limit));
                 tc_fence_after();
                 if (warp == kFirstEpiWarp && lane == 0) SPARQ_PROF_TL(1, 2 * wt, cta_t0);
                 pre_full = 0;
@@ -606,7 +607,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 staged_nt = nt;
                 epi_stage_scale_bias<kEpi>(g, nt * BN, BN, et, s_scale, s_bias);
             }
-            SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status));
+            SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status, g.wait_limit));
             tc_fence_after();
             const int oh = ((int)walk.tin + j) * g.TR + tr;
             const bool row_ok = slot_ok && (oh < g.Ho);
@@ -634,7 +635,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             const int b = rb;
             const uint32_t wph = ruse & 1u;
             for (int j = 0; j < g.G; ++j) {
-                SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), wph, abort_flag, g.status));
+                SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), wph, abort_flag, g.status, g.wait_limit));
                 if (warp == kFirstXfWarp && lane == 0 && gi == 0) SPARQ_PROF_TL(2, 2 * j, cta_t0);
                 if (j < (int)walk.cnt) {
                     const uint32_t nvec = piece_len(j) >> 4;

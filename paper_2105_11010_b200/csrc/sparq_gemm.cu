@@ -15,7 +15,8 @@ __device__ long long g_prof[148 * 16];
 __device__ long long g_prof_tl[4 * 64];
 #endif
 
-void release_gemm_state() {}
+// Limit of the device-side waits of every fused launch, in SM cycles.
+static long long g_wait_limit = kWaitLimitCycles;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -51,6 +52,13 @@ struct MapSlot { bool used; MapKey key; CUtensorMap map; };
 constexpr int kMapSlots = 256;
 static MapSlot g_map_cache[kMapSlots];
 static std::mutex g_map_mutex;
+
+// Forgets the cached tensor maps (host memory only; they are re-encoded on demand).
+void release_gemm_state()
+{
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    for (MapSlot &s : g_map_cache) s.used = false;
+}
 
 static unsigned map_hash(const MapKey &k)
 {
@@ -225,44 +233,23 @@ static int fill_common(GemmArgs *g, const XformArgs &x, const sparq_epilogue *e,
     g->f32_out = e->f32_out;
     g->u8_out = e->u8_out;
     g->status = status;
+    g->wait_limit = g_wait_limit;
     g->residual = e->residual;
     g->residual_scale = e->residual_scale;
     return next_transform_args(e, g->N, &g->next_mode, &g->next_rnd, &g->next_xf);
 }
 
+int gemm_with_status(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb, int64_t M, int64_t N, int64_t K,
+                     const XformArgs &x, const sparq_epilogue *e, unsigned int *status, cudaStream_t st);
+
+// The fused GEMM with the library's own status word (allocated on first use).
 static int gemm_impl(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb, int64_t M, int64_t N, int64_t K,
                      const XformArgs &x, const sparq_epilogue *e, cudaStream_t st)
 {
-    int sms = 0;
-    int rc = device_info(&sms);
-    if (rc != SPARQ_OK) return rc;
     unsigned int *status = nullptr;
-    rc = get_status_word(&status);
+    int rc = get_status_word(&status);
     if (rc != SPARQ_OK) return rc;
-
-    // reduction step: the one that pads K the least; ties go to the wider step
-    const int64_t pad128 = (K + 127) / 128 * 128, pad64 = (K + 63) / 64 * 64;
-    const int bk = (pad64 < pad128) ? 64 : 128;
-    const int bn = pick_bn(M, N, sms, x.mode != SPARQ_MODE_NONE);
-
-    CUtensorMap ma, mb;
-    rc = encode_2d(&ma, A, K, M, lda, bk, kBM);
-    if (rc != SPARQ_OK) return rc;
-    rc = encode_2d(&mb, B, K, N, ldb, bk, bn);
-    if (rc != SPARQ_OK) return rc;
-
-    GemmArgs g;
-    memset(&g, 0, sizeof(g));
-    g.M = M; g.N = N; g.K = K;
-    g.k_blocks = (int)((K + bk - 1) / bk);
-    rc = fill_common(&g, x, e, status);
-    if (rc != SPARQ_OK) return rc;
-    const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
-    if (tiles >= ((int64_t)1 << 31)) return set_error(SPARQ_ERR_UNSUPPORTED, "more than 2^31 output tiles");
-    const int grid = (int)(tiles < sms ? tiles : sms);
-    cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
-    if (ce != cudaSuccess) return cuda_error(ce, "sparq_gemm_kernel launch");
-    return SPARQ_OK;
+    return gemm_with_status(A, lda, B, ldb, M, N, K, x, e, status, st);
 }
 
 // NHWC activation tensor read as a box of cb channels x wp columns x rows input rows of one
@@ -425,6 +412,7 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     g.scale = e->scale; g.bias = e->bias; g.relu = e->relu ? 1 : 0; g.inv_out_scale = e->inv_out_scale;
     g.acc_out = e->acc_out; g.f32_out = e->f32_out; g.u8_out = e->u8_out;
     g.status = status;
+    g.wait_limit = g_wait_limit;
     g.residual = e->residual;
     g.residual_scale = e->residual_scale;
     rc = next_transform_args(e, g.N, &g.next_mode, &g.next_rnd, &g.next_xf);
@@ -438,8 +426,8 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     return 1;
 }
 
-// The same launch as gemm_impl for callers that bring their own status word (a device
-// pointer) instead of the library-allocated one.  Nothing here allocates device memory.
+// Tile choice, tensor maps and launch of the fused GEMM.  The caller brings the status word (a
+// device pointer); nothing here allocates device memory.
 int gemm_with_status(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb, int64_t M, int64_t N, int64_t K,
                      const XformArgs &x, const sparq_epilogue *e, unsigned int *status, cudaStream_t st)
 {
@@ -447,7 +435,7 @@ int gemm_with_status(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     int rc = device_info(&sms);
     if (rc != SPARQ_OK) return rc;
     const int64_t pad128 = (K + 127) / 128 * 128, pad64 = (K + 63) / 64 * 64;
-    const int bk = (pad64 < pad128) ? 64 : 128;
+    const int bk = (pad64 < pad128) ? 64 : 128;   // the step that pads K the least; ties go to the wider one
     const int bn = pick_bn(M, N, sms, x.mode != SPARQ_MODE_NONE);
     CUtensorMap ma, mb;
     rc = encode_2d(&ma, A, K, M, lda, bk, kBM);

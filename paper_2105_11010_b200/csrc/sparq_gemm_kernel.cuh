@@ -45,6 +45,8 @@ constexpr int kGemmThreads = 32 * (kFirstXfWarp + kNumXfWarps);
 // Epilogue warps of a kernel instantiated for `mode`.
 __host__ __device__ constexpr int epi_warps(int mode) { return mode == SPARQ_MODE_NONE ? kNumEpiWarps + kNumXfWarps : kNumEpiWarps; }
 constexpr int kSmemBudget = 200 * 1024;  // for the stage ring
+// Default limit of every device-side wait, in SM clock cycles (about a second).  The limit is a
+// kernel argument, so that a diagnostic launch can make a wait run out in microseconds.
 constexpr long long kWaitLimitCycles = 2000000000LL;
 
 // Optional per-role cycle counters (builds with -DSPARQ_PROF -rdc=true only): how long each warp role
@@ -86,6 +88,7 @@ struct GemmArgs {
     float *f32_out;
     uint8_t *u8_out;
     unsigned int *status;
+    long long wait_limit;   // cycles after which a device-side wait gives up
     // producer-side transform of u8_out (mode NONE = off)
     int next_mode, next_rnd;
     XformDev next_xf;
@@ -163,7 +166,7 @@ __device__ __forceinline__ uint32_t mbar_test3(uint32_t bar0, uint32_t parity0, 
 // Bounded wait.  Returns false (after flagging) if the phase did not complete in time or
 // if another thread of the CTA already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          unsigned int *status, bool ignore_abort = false)
+                                          unsigned int *status, long long limit_cycles, bool ignore_abort = false)
 {
     if (mbar_try_wait(bar, parity)) return true;
     if (!ignore_abort && *abort_flag) return false;
@@ -172,7 +175,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 0x3FFu) == 0) {
             if (!ignore_abort && *abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1u;
                 atomicOr(status, 1u);
                 return false;
@@ -771,7 +774,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 for (int kb = 0; kb < kb_count; ++kb, ++it) {
                     const int s = it % S;
                     const uint32_t use = it / S;
-                    if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_empty[s]), (use - 1) & 1, abort_flag, g.status));
+                    if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_empty[s]), (use - 1) & 1, abort_flag, g.status, g.wait_limit));
                     if (*abort_flag) break;   // stop issuing copies once the CTA has given up
                     const uint32_t full = smem_u32(&bar_full[s]);
                     mbar_expect_tx(full, Cfg::kStageBytes);
@@ -793,7 +796,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             if (*abort_flag) {
                 const uint32_t first = it > (uint32_t)S ? it - S : 0;
                 for (uint32_t j = first; j < it; ++j)
-                    mbar_wait(smem_u32(&bar_full[j % S]), (j / S) & 1, abort_flag, g.status, true);
+                    mbar_wait(smem_u32(&bar_full[j % S]), (j / S) & 1, abort_flag, g.status, g.wait_limit, true);
             }
         }
         __syncwarp();
@@ -815,12 +818,12 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
                 const int acc = local_tile & 1;
                 const uint32_t acc_use = local_tile >> 1;
-                if (acc_use > 0) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status));
+                if (acc_use > 0) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status, g.wait_limit));
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 for (int kb = 0; kb < kb_count; ++kb) {
-                    if (MODE == SPARQ_MODE_NONE) SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_full[s]), ph, abort_flag, g.status));
-                    else SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_xf[s]), ph, abort_flag, g.status));
+                    if (MODE == SPARQ_MODE_NONE) SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_full[s]), ph, abort_flag, g.status, g.wait_limit));
+                    else SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_xf[s]), ph, abort_flag, g.status, g.wait_limit));
                     tc_fence_after();
                     const uint64_t st_off = (uint64_t)((uint32_t)s * (uint32_t)(Cfg::kStageBytes >> 4));
                     const uint64_t adesc = adesc0 + st_off, bdesc = bdesc0 + st_off;
@@ -838,7 +841,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             SPARQ_PROF_STORE(4, SPARQ_PROF_NOW() - mt0);
             // all tensor-core work of this CTA has retired before tensor memory is freed
             tc_commit_if(smem_u32(&bar_done), elected);
-            mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, true);
+            mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, g.wait_limit, true);
         }
         __syncwarp();
     } else if (warp < kFirstEpiWarp + epi_warps(MODE)) {
@@ -864,7 +867,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 const int64_t row = (int64_t)tile * kBM + quarter * 32 + lane;    // one column tile: row tile = tile
                 const bool row_ok = row < g.M;
                 const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + team * BN + (uint32_t)tcbase;
-                SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[team]), (local_tile >> 1) & 1u, abort_flag, g.status));
+                SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[team]), (local_tile >> 1) & 1u, abort_flag, g.status, g.wait_limit));
                 tc_fence_after();
 #pragma unroll 1
                 for (int ch = 0; ch < kTeamCols / 32; ++ch) {
@@ -892,7 +895,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 staged_nt = nt;
                 epi_stage_scale_bias<kEpi>(g, nt * BN, BN, et, s_scale, s_bias);
             }
-            SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status));
+            SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status, g.wait_limit));
             tc_fence_after();
             const int64_t row = mt * kBM + quarter * 32 + lane;
             const bool row_ok = row < g.M;
@@ -922,7 +925,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             for (int kb = 0; kb < kb_count; ++kb, ++it) {
                 if ((int)(it & 1u) != team) continue;      // the other team's stage
                 const int s = it % S;
-                SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_full[s]), (it / S) & 1, abort_flag, g.status));
+                SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_full[s]), (it / S) & 1, abort_flag, g.status, g.wait_limit));
                 const uint32_t base = a_stage(s) + (uint32_t)xt * 16u;
 #pragma unroll
                 for (int j0 = 0; j0 < kPerThread; j0 += kBatch) {

@@ -44,6 +44,17 @@ int scratch_base(unsigned char **base)
 }
 
 }  // namespace
+
+// Device address of the status word inside the static scratch (no allocation).
+int static_status_word(unsigned int **dptr)
+{
+    unsigned char *base = nullptr;
+    int rc = scratch_base(&base);
+    if (rc != SPARQ_OK) return rc;
+    *dptr = reinterpret_cast<unsigned int *>(base);
+    return SPARQ_OK;
+}
+
 }  // namespace sparq
 
 using namespace sparq;
