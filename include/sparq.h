@@ -15,8 +15,11 @@
  *     validates its arguments on the host, enqueues its kernels on `stream` and returns
  *     without synchronizing.
  *   - Return value: SPARQ_OK (0) or a negative sparq_status.  On error nothing has been
- *     enqueued and sparq_last_error() describes the reason.  No entry point throws,
- *     aborts or traps the device.
+ *     enqueued and sparq_last_error() describes the reason (the entry points that enqueue
+ *     more than one kernel -- the host-buffer forms, sparq_gemm_s8_static,
+ *     sparq_gemm_s8_sparse24 -- may have enqueued their earlier kernels when a later launch
+ *     fails; their outputs are then undefined).  No entry point throws, aborts or traps the
+ *     device.
  *   - The library is thread-compatible: concurrent calls are allowed, the error string
  *     is per host thread.
  */
@@ -196,7 +199,13 @@ SPARQ_API int sparq_conv2d_nhwc_s8_host(const uint8_t *x_host, int n, int h, int
  *     SPARQ_ERR_UNSUPPORTED with the limit in sparq_last_error().  Other requirements as
  *     for sparq_gemm_s8.
  *   - The first call on a device looks up the array's device address (set-up, once per
- *     device, with that device current).  Make that first call outside any stream capture.
+ *     device, with that device current).  Like the first use of any kernel of a library,
+ *     it also makes the CUDA runtime load the library's device code, and the driver
+ *     reserves the array's SPARQ_STATIC_SCRATCH_BYTES then: memory taken by the driver for
+ *     the code image, not an allocation this entry point makes, but it does come out of
+ *     the device's free memory at that moment.  So make one call at start-up, before the
+ *     host's own pool claims the device, and outside any stream capture; every later call
+ *     leaves the free device memory exactly as it found it.
  *   - The call is synchronous: it returns after `stream` has drained, so the outputs are
  *     complete and a device-side timeout is reported by this call (SPARQ_ERR_TIMEOUT),
  *     not by sparq_check.
@@ -245,8 +254,8 @@ SPARQ_API int sparq_unpack(const uint8_t *data, const uint8_t *ctrl, size_t rows
                  const sparq_params *p, uint8_t *out, void *stream);
 
 /* ---- Uniform min-max quantization (Section 5) ----------------------------------------------
- * The paper's models are quantized "using a simple uniform min-max quantization": unsigned
- * symmetric per layer for activations, signed symmetric per kernel for weights, with the
+ * Section 5: the paper's models are quantized uniformly from min-max statistics, unsigned
+ * symmetric per layer for activations and signed symmetric per kernel for weights, with the
  * statistics gathered over a few calibration batches.  These three calls are that front
  * end on the device; the data set and the calibration run are the caller's.
  * x is fp32 (SPARQ_DTYPE_F32) or bf16 (SPARQ_DTYPE_BF16, widened exactly), 16-byte aligned,
@@ -315,12 +324,34 @@ SPARQ_API int sparq_gemm_s8_sparse24(const uint8_t *A, const int8_t *w_exp, int6
  * bad coordinates, or SPARQ_ERR_CUDA if the stream is in error. */
 SPARQ_API int sparq_check(void *stream);
 
+/* Diagnostic: launches a one-CTA kernel that waits, with a limit of `limit_cycles` SM clock
+ * cycles (1e3 .. 1e8), on a barrier that nothing ever completes, using the wait, abort-flag
+ * and tensor-memory code of the fused kernels (whose own limit is about a second and whose
+ * barriers always complete, so their give-up path cannot be reached on demand).  The kernel
+ * always returns normally; afterwards sparq_check(stream) reports SPARQ_ERR_TIMEOUT once and
+ * SPARQ_OK from then on, and every other entry point keeps working.  With use_static_word
+ * the bit is recorded in sparq_gemm_s8_static's own status word instead, which the next
+ * call of that entry point reports and clears.  report: 4 words on the DEVICE -- the first
+ * wait gave up (1), a second wait with a 1000x longer limit left through the CTA's abort
+ * flag (1), the cycles that second wait spent, the kernel reached its end (1).  The paper has
+ * no counterpart. */
+SPARQ_API int sparq_selftest_wait_timeout(int64_t limit_cycles, int use_static_word, uint32_t *report, void *stream);
+
+/* Diagnostic: the tensor core's own rate, the ceiling the fused kernels are measured against.
+ * One CTA per SM issues iters x 4 tcgen05.mma kind::i8 instructions of 128 x bn x 32
+ * (u8 x s8 -> s32; bn = 64, 128 or 256; iters <= 1e6) on operands resident in shared memory,
+ * with no global-memory traffic, transform or epilogue, and writes the SM-clock cycles from
+ * its first issue to the retirement of its last MMA to cycles_out[cta] (DEVICE, one int64 per
+ * SM).  MACs per launch = SMs * iters * 4 * 128 * bn * 32.  Returns the number of CTAs
+ * launched (> 0) or a negative sparq_status.  The paper has no counterpart. */
+SPARQ_API int sparq_selftest_mma_rate(int bn, int iters, int64_t *cycles_out, void *stream);
+
 /* Text of the calling thread's most recent error ("" if none).  The pointer stays valid
  * until the thread's next failing call. */
 SPARQ_API const char *sparq_last_error(void);
 
-/* Releases what the library itself holds on the current device (cached descriptors, the
- * status word).  Safe to call more than once; later calls re-create what they need. */
+/* Releases what the library itself holds on the current device (the status word, the
+ * host-buffer forms' staging buffers) and forgets the cached tensor-map encodings.  Safe to call more than once; later calls re-create what they need. */
 SPARQ_API int sparq_shutdown(void);
 
 #ifdef __cplusplus

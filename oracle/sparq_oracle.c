@@ -437,10 +437,9 @@ void oracle_epilogue(const int32_t *acc, int64_t M, int64_t N,
 
 /* ---- Section 5: uniform min-max quantization of the network's tensors ------ */
 
-/* The paper quantizes every layer "using a simple uniform min-max quantization, employing
- * symmetric unsigned per-layer quantization for activations and symmetric signed
- * per-kernel quantization for weights" (Section 5).  The statistic of both is the largest
- * magnitude; NaNs are skipped.  bf16 inputs are given as their 16-bit patterns and widened
+/* Section 5: every layer is quantized uniformly from its min-max statistics -- activations
+ * unsigned and symmetric with one scale per layer, weights signed and symmetric with one
+ * scale per kernel.  The statistic of both is the largest magnitude; NaNs are skipped.  bf16 inputs are given as their 16-bit patterns and widened
  * exactly (bf16 is the top half of an fp32). */
 static float load_elem(const void *x, int is_bf16, size_t i)
 {

@@ -19,5 +19,5 @@ from ._binding import (  # noqa: F401
     sparq_sparse24_expanded_k, sparq_sparse24_expand_weights, sparq_sparse24_expand_activations,
     sparq_gemm_s8_sparse24,
     sparq_absmax, sparq_quantize_act_u8, sparq_quantize_weight_s8, DTYPE_F32, DTYPE_BF16,
-    sparq_check, sparq_last_error, sparq_shutdown,
+    sparq_check, sparq_last_error, sparq_shutdown, sparq_selftest_wait_timeout, sparq_selftest_mma_rate,
 )

@@ -107,6 +107,10 @@ def load_library() -> ctypes.CDLL:
         L.sparq_conv2d_nhwc_s8_host.restype = i32
         L.sparq_gemm_s8_static.argtypes = L.sparq_gemm_s8.argtypes
         L.sparq_gemm_s8_static.restype = i32
+        L.sparq_selftest_wait_timeout.argtypes = [i64, i32, vp, vp]
+        L.sparq_selftest_wait_timeout.restype = i32
+        L.sparq_selftest_mma_rate.argtypes = [i32, i32, vp, vp]
+        L.sparq_selftest_mma_rate.restype = i32
         L.sparq_check.argtypes = [vp]
         L.sparq_check.restype = i32
         L.sparq_last_error.argtypes = []
@@ -148,6 +152,26 @@ def sparq_last_error() -> str:
 
 def sparq_check(stream=None) -> None:
     _raise(load_library().sparq_check(_stream_ptr(stream)))
+
+
+def sparq_selftest_wait_timeout(limit_cycles: int, report: torch.Tensor, use_static_word: bool = False,
+                                stream=None) -> None:
+    """Diagnostic launch whose bounded wait runs out; ``report`` is 4 int32/uint32 words on the device."""
+    if report.numel() < 4 or report.element_size() != 4 or not report.is_cuda:
+        raise ValueError("report must hold four 32-bit words on the device")
+    _raise(load_library().sparq_selftest_wait_timeout(int(limit_cycles), int(bool(use_static_word)),
+                                                      report.data_ptr(), _stream_ptr(stream)))
+
+
+def sparq_selftest_mma_rate(bn: int, iters: int, cycles_out: torch.Tensor, stream=None) -> int:
+    """MMA-only loop on every SM; ``cycles_out`` (int64, one per SM, device) receives each CTA's cycles.
+    Returns the number of CTAs launched."""
+    if cycles_out.dtype != torch.int64 or not cycles_out.is_cuda or cycles_out.numel() < 256:
+        raise ValueError("cycles_out must be an int64 device tensor of at least 256 elements")
+    rc = load_library().sparq_selftest_mma_rate(int(bn), int(iters), cycles_out.data_ptr(), _stream_ptr(stream))
+    if rc < 0:
+        _raise(rc)
+    return rc
 
 
 def sparq_shutdown() -> None:

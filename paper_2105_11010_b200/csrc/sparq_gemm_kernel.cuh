@@ -173,7 +173,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 0x3FFu) == 0) {
+        if ((it & 0x3Fu) == 0) {
             if (!ignore_abort && *abort_flag) return false;
             if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1u;

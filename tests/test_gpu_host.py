@@ -5,6 +5,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import sparq_synth as synth
 import paper_2105_11010_b200 as sparq
 
@@ -47,6 +48,11 @@ def test_conv_host_chunked_equals_device():
                                         u8_out=h["u8"], residual=pinned(res), residual_scale=0.25)
         for k in h:
             assert torch.equal(h[k], d[k].cpu()), k
+    # and against the oracle directly
+    acc = oracle.conv2d_nhwc(x, w, (1, 1), (1, 1), VS.mode, 4, 0x1F, 1)
+    f, q = oracle.epilogue(acc, scale, bias, True, inv, residual=res, residual_scale=0.25)
+    assert np.array_equal(h["acc"].numpy(), acc) and np.array_equal(h["u8"].numpy(), q)
+    assert np.allclose(h["f32"].numpy(), f, rtol=1e-6, atol=1e-6)
 
 
 def test_gemm_host_chunked_equals_device():
@@ -65,3 +71,13 @@ def test_gemm_host_chunked_equals_device():
                              f32_out=h_f, u8_out=h_q)
     assert torch.equal(h_f, d_f.cpu())
     assert torch.equal(h_q, d_q.cpu())
+    f, q = oracle.epilogue(oracle.gemm(A, B, VS.mode, 4, 0x1F, 1), scale, None, True, inv)
+    assert np.array_equal(h_q.numpy(), q) and np.allclose(h_f.numpy(), f, rtol=1e-6, atol=1e-6)
+
+
+def test_quantize_host_equals_oracle():
+    rows, row_len = 3001, 1000
+    x = synth.activations(960, (rows, row_len), 0.5)
+    out = torch.zeros((rows, row_len), dtype=torch.uint8).pin_memory()
+    sparq.sparq_quantize_host(pinned(x), out, rows, row_len, VS)
+    assert np.array_equal(out.numpy(), oracle.transform(x, VS.mode, 4, 0x1F, 1))
