@@ -1,16 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the SPARQ hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras] [--full]
+                    [--section NAME]
 
-A step is one pass of the whole hot path -- vSPARQ transform (n = 4, five placements,
-round to nearest), u8 x s8 -> s32 implicit-GEMM convolution, fp32 scale + bias + ReLU +
-requantize to uint8 -- over one batch of the ResNet-18-style workload
-(32 x 56 x 56 x 64 NHWC uint8 activations with 45 % zeros, 64 filters of 3x3, stride 1,
-pad 1).  One fused kernel launch per step.  Prints one JSON line.
+A step is one pass of the whole hot path -- vSPARQ transform (n = 4, five placements, round to
+nearest) inside the u8 x s8 -> s32 implicit-GEMM convolution, fp32 scale + bias + ReLU +
+requantize to uint8 -- over one batch of the largest single-GPU workload of the ablation config:
+128 x 28 x 28 x 128 NHWC uint8 activations (50 % zeros) -> 128 filters of 3x3, stride 1, pad 1
+(29.6 GOP).  One fused kernel launch per step.  Prints ONE JSON line; the other configs (tiny
+GEMM, ResNet-18 layer, ResNet-50 sweep, 2^30-byte transform, the ablation grid) are compact
+entries of its `extra` object, and `--section NAME` prints one of them in full.
 
-With --impl reference the CPU oracle is timed instead (rank 0 only): each step is the
-same layer on a bounded number of images.
+With --impl reference the CPU oracle is timed instead (rank 0 only): each step is the same layer
+on a bounded number of images.
 """
 from __future__ import annotations
 
@@ -33,33 +36,39 @@ import sparq_synth as synth  # noqa: E402
 METRIC = "fused SPARQ INT8 conv TOPS"
 UNIT = "TOPS"
 
-# ResNet-18-style layer the metric is quoted on
-NB, H, W, C, COUT, R, S, STRIDE, PAD = 32, 56, 56, 64, 64, 3, 3, 1, 1
-ZERO_FRAC = 0.45
-SEED = 1
-OPS_PER_STEP = 2 * NB * H * W * COUT * R * S * C          # dense count: no MAC is skipped
-IN_BYTES = NB * H * W * C
-OUT_BYTES = NB * H * W * COUT
-WGT_BYTES = COUT * R * S * C
+# the layer the headline is quoted on (ablation config, fused vSPARQ 5opt +R, 50 % zeros)
+HEAD = dict(nb=128, h=28, w=28, c=128, cout=128, r=3, s=3, stride=1, pad=1, zf=0.5, seed=500)
+# ResNet-18-style layer (32 x 56 x 56 x 64 -> 64, 45 % zeros)
+RN18 = dict(nb=32, h=56, w=56, c=64, cout=64, r=3, s=3, stride=1, pad=1, zf=0.45, seed=1)
 L2_BYTES = 126 * 1024 * 1024
+OPS_PER_STEP = 2 * 128 * 28 * 28 * 128 * 3 * 3 * 128       # the headline layer; dense count: no MAC is skipped
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
-INT8_OVER_BF16 = 2.0     # nominal dense ratio (4.5 POPS int8 vs 2.25 PFLOPS bf16)
-CONV_TRAFFIC_BYTES = 6541824 + 0   # ncu dram read + write bytes per launch; set to None whenever the kernel changes
-# transform kernel (bSPARQ, n=4, 5opt, +R) captured on 2^28 activations: 268,445,184 B read +
-# 214,811,392 B written (the rest of the output is still dirty in L2); scales with the count
-TRANSFORM_TRAFFIC_PER_2P28 = 268445184 + 214811392
-# fused GEMM kernel on the 56x56x64 -> 256 layer at batch 64: 12.92 MB read, 2.0 MB written per launch (most of
-# the 51 MB output is still dirty in L2 when the launch ends); None whenever that kernel changes
-LAYER1X1_TRAFFIC_BYTES = 12924928 + 2003200
+NOMINAL_INT8_TOPS = 4500.0          # dense, datasheet (2 x the 2.25 PFLOP/s bf16 figure)
+MIN_TIMED_MS = 50.0                 # device time every reported figure is the median over, at least
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarized under
+# profiles/; None whenever the kernel has changed since its capture.
+TRAFFIC = {"head": None, "rn18": None, "layer1x1": None, "transform_per_2p28": 268445184 + 214811392}
+
+
+def ops_of(L):
+    ho = (L["h"] + 2 * L["pad"] - L["r"]) // L["stride"] + 1
+    wo = (L["w"] + 2 * L["pad"] - L["s"]) // L["stride"] + 1
+    return 2 * L["nb"] * ho * wo * L["cout"] * L["r"] * L["s"] * L["c"]
+
+
+def bytes_of(L):
+    ho = (L["h"] + 2 * L["pad"] - L["r"]) // L["stride"] + 1
+    wo = (L["w"] + 2 * L["pad"] - L["s"]) // L["stride"] + 1
+    return L["nb"] * L["h"] * L["w"] * L["c"], L["nb"] * ho * wo * L["cout"], L["cout"] * L["r"] * L["s"] * L["c"]
 
 
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         p = json.load(open(path))
-        return dict(hbm=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops"]),
-                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
-    return dict(hbm=FALLBACK_HBM_GBS, bf16=FALLBACK_BF16_TFLOPS, bf16_sustained=1400.0, source="fallback")
+        return dict(hbm=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops"]), source="measured")
+    return dict(hbm=FALLBACK_HBM_GBS, bf16=FALLBACK_BF16_TFLOPS, source="fallback")
 
 
 class ClockSampler:
@@ -80,7 +89,7 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100", "-i", str(self.gpu_index)],
+                 "-lms", "50", "-i", str(self.gpu_index)],
                 stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -115,20 +124,10 @@ class ClockSampler:
         return out
 
 
-def build_layer(device, sets):
-    """`sets` independent input / output buffer pairs (rotated so that consecutive steps
-    never find their operands in L2) and the resident layer parameters."""
-    import torch
-    xs = [torch.from_numpy(synth.activations(SEED, (NB, H, W, C), ZERO_FRAC, stream=10 + i)).to(device)
-          for i in range(sets)]
-    outs = [torch.empty((NB, H, W, COUT), dtype=torch.uint8, device=device) for _ in range(sets)]
-    wt = torch.from_numpy(synth.weights(SEED, (COUT, R, S, C))).to(device)
-    scale = torch.from_numpy(synth.scales(SEED, COUT)).to(device)
-    bias = torch.from_numpy(synth.bias(SEED, COUT)).to(device)
-    return xs, outs, wt, scale, bias
-
+# ---- timing ------------------------------------------------------------------------------------
 
 def time_region(fn, steps, warmup, sync):
+    """Eager loop, CUDA events on the current stream (for kernels that take >= 100 us)."""
     import torch
     for i in range(warmup):
         fn(i)
@@ -142,26 +141,168 @@ def time_region(fn, steps, warmup, sync):
     return e0.elapsed_time(e1)      # ms
 
 
-def time_graph(fn, steps, warmup, sync):
-    """Device time of `steps` calls captured in one CUDA graph (ms): the calls are enqueued
-    by the graph, not by Python, whose ~15 us per call would otherwise hide any kernel
-    shorter than that.  One untimed replay first (it uploads the graph)."""
+class GraphTimer:
+    """`steps` calls captured once into a CUDA graph (Python needs ~15 us to enqueue one call,
+    more than a small layer takes on the device).  Each replay runs exactly `steps` steps and
+    is timed by its own event pair on the launching stream; replays are enqueued back to back
+    until at least `min_ms` of device time has been covered, and the median replay is reported."""
+
+    def __init__(self, fn, steps, warmup):
+        import torch
+        self.steps = steps
+        for i in range(warmup):
+            fn(i)
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            for i in range(steps):
+                fn(warmup + i)
+        self.graph.replay()            # the first replay also uploads the graph
+        torch.cuda.synchronize()
+        self.replays = 0
+
+    def run(self, min_ms=MIN_TIMED_MS, barrier=None):
+        import torch
+        probe0, probe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        probe0.record(); self.graph.replay(); probe1.record()
+        torch.cuda.synchronize()
+        one = max(probe0.elapsed_time(probe1), 1e-3)
+        n = int(min(2000, max(5, np.ceil(min_ms / one))))
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+        ev[0].record()
+        for i in range(n):
+            self.graph.replay()
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+        times = [ev[i].elapsed_time(ev[i + 1]) for i in range(n)]
+        self.replays = n
+        return statistics.median(times) / self.steps, sum(times), n
+
+
+def device_activations(device, shape, zf, seed):
+    """The config's value recipe drawn on the device (seeded torch generator): zeros with
+    probability zf, else clip(round(|N(0,1)| * 40), 1, 255)."""
     import torch
-    for i in range(warmup):
-        fn(i)
-    sync()
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph):
-        for i in range(steps):
-            fn(warmup + i)
-    graph.replay()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sync()
-    e0.record()
-    graph.replay()
-    e1.record()
-    sync()
-    return e0.elapsed_time(e1)
+    g = torch.Generator(device=device).manual_seed(seed)
+    n = int(np.prod(shape))
+    z = torch.randn(n, generator=g, device=device)
+    v = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
+    if zf > 0:
+        v[torch.rand(n, generator=g, device=device) < zf] = 0
+    return v.view(*shape)
+
+
+class ConvLayer:
+    """One convolution workload with `sets` rotating input / output buffer pairs, so that
+    consecutive steps never find their operands in the 126 MiB L2."""
+
+    def __init__(self, device, L, sets=None, host_recipe=False):
+        import torch
+        self.L = L
+        in_b, out_b, _ = bytes_of(L)
+        if sets is None:
+            sets = max(2, min(24, int(1.3 * L2_BYTES // (in_b + out_b)) + 1))
+        self.sets = sets
+        ho = (L["h"] + 2 * L["pad"] - L["r"]) // L["stride"] + 1
+        wo = (L["w"] + 2 * L["pad"] - L["s"]) // L["stride"] + 1
+        shape = (L["nb"], L["h"], L["w"], L["c"])
+        if host_recipe:
+            self.xs = [torch.from_numpy(synth.activations(L["seed"], shape, L["zf"], stream=10 + i)).to(device)
+                       for i in range(sets)]
+        else:
+            self.xs = [device_activations(device, shape, L["zf"], L["seed"] * 64 + i) for i in range(sets)]
+        self.outs = [torch.empty((L["nb"], ho, wo, L["cout"]), dtype=torch.uint8, device=device) for _ in range(sets)]
+        self.wt = torch.from_numpy(synth.weights(L["seed"], (L["cout"], L["r"], L["s"], L["c"]))).to(device)
+        self.scale = torch.from_numpy(synth.scales(L["seed"], L["cout"])).to(device)
+        self.bias = torch.from_numpy(synth.bias(L["seed"], L["cout"])).to(device)
+        self.inv = synth.inv_out_scale(L["r"] * L["s"] * L["c"], L["zf"])
+        self.scratch = None
+
+    def fused(self, params):
+        import paper_2105_11010_b200 as sparq
+        L = self.L
+
+        def step(i):
+            j = i % self.sets
+            sparq.sparq_conv2d_nhwc_s8(self.xs[j], self.wt, (L["stride"], L["stride"]), (L["pad"], L["pad"]), params,
+                                       scale=self.scale, bias=self.bias, relu=True, inv_out_scale=self.inv,
+                                       u8_out=self.outs[j])
+        return step
+
+    def unfused(self, params):
+        """Separate transform kernel into a scratch tensor, then the plain A8W8 convolution."""
+        import torch
+        import paper_2105_11010_b200 as sparq
+        L = self.L
+        if self.scratch is None:
+            self.scratch = [torch.empty_like(self.xs[0]) for _ in range(min(self.sets, 4))]
+        none = sparq.SparqParams(sparq.MODE_NONE)
+        rows, row_len = L["nb"] * L["h"] * L["w"], L["c"]
+
+        def step(i):
+            j = i % self.sets
+            t = self.scratch[i % len(self.scratch)]
+            sparq.sparq_quantize(self.xs[j], t, rows, row_len, params)
+            sparq.sparq_conv2d_nhwc_s8(t, self.wt, (L["stride"], L["stride"]), (L["pad"], L["pad"]), none,
+                                       scale=self.scale, bias=self.bias, relu=True, inv_out_scale=self.inv,
+                                       u8_out=self.outs[j])
+        return step
+
+
+def roofline_tensor(ops, ms, mma, pk, clocks_mhz, traffic, kernel, alg_bytes):
+    """Roofline object of a contraction: achieved TOP/s of one step in a back-to-back stream
+    against the measured tcgen05.mma kind::i8 rate at the SM clock sampled during the run."""
+    tops = ops / (ms * 1e-3) / 1e12
+    clk = clocks_mhz or pk.get("sm_max_mhz") or 1965.0
+    peak = mma["mac_per_clk_sm"] * mma["sms"] * 2 * clk * 1e6 / 1e12 if mma else pk["bf16"] * 2
+    return {
+        "bound": "tensor", "achieved": round(tops, 1), "peak": round(peak, 1), "unit": "TOP/s",
+        "frac": round(tops / peak, 4), "traffic": traffic,
+        "peak_source": (f"own MMA-only kind::i8 loop: {mma['mac_per_clk_sm']:.0f} MAC/clk/SM x {mma['sms']} SMs x "
+                        f"{clk:.0f} MHz sampled" if mma else f"{pk['source']} bf16 burst x 2"),
+        "frac_of_2x_bf16_burst": round(tops / (pk["bf16"] * 2), 4),
+        "frac_of_nominal_4500": round(tops / NOMINAL_INT8_TOPS, 4),
+        "timing": "median CUDA-graph replay / steps: per step in a back-to-back stream (a launch's prologue overlaps "
+                  "its predecessor's tail), not per isolated launch",
+        "kernel": kernel, "algorithmic_ops_per_launch": ops, "algorithmic_bytes_per_launch": alg_bytes,
+        "hbm_floor_ms": round(alg_bytes / (pk["hbm"] * 1e9) * 1e3, 5),
+    }
+
+
+# ---- sections ------------------------------------------------------------------------------------
+
+def mma_peak_section(device, bns=(64, 128, 256), iters=4000):
+    """The tensor core's own rate: the library's MMA-only loop on every SM (operands resident in
+    shared memory).  MAC/clk/SM from the slowest CTA's cycle count; TOP/s from CUDA events."""
+    import torch
+    import paper_2105_11010_b200 as sparq
+    cyc = torch.zeros(256, dtype=torch.int64, device=device)
+    out = {}
+    for bn in bns:
+        for _ in range(2):
+            sms = sparq.sparq_selftest_mma_rate(bn, iters, cyc)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        sms = sparq.sparq_selftest_mma_rate(bn, iters, cyc)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        worst = int(cyc[:sms].max().item())
+        macs_cta = iters * 4 * 128 * bn * 32
+        out[f"n{bn}"] = {"mac_per_clk_sm": round(macs_cta / worst, 1), "ms": round(ms, 4),
+                         "tops_by_events": round(2 * macs_cta * sms / ms / 1e9, 1)}
+    sparq.sparq_check()
+    best = max(out.values(), key=lambda d: d["mac_per_clk_sm"])
+    out["sms"] = sms
+    out["mac_per_clk_sm"] = best["mac_per_clk_sm"]
+    out["implied_mhz"] = round(best["tops_by_events"] * 1e12 / (2 * best["mac_per_clk_sm"] * sms) / 1e6, 0)
+    return out
 
 
 def transform_section(device, pk, n, steps, warmup):
@@ -170,25 +311,23 @@ def transform_section(device, pk, n, steps, warmup):
     import torch
     import paper_2105_11010_b200 as sparq
     sync = torch.cuda.synchronize
-    gen = torch.Generator(device=device).manual_seed(4)
     x = torch.empty(n, dtype=torch.uint8, device=device)
     chunk = min(n, 1 << 26)
-    for lo in range(0, n, chunk):
-        z = torch.randn(chunk, generator=gen, device=device)
-        v = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
-        v[torch.rand(chunk, generator=gen, device=device) < 0.5] = 0
-        x[lo:lo + chunk] = v
+    for k, lo in enumerate(range(0, n, chunk)):
+        x[lo:lo + chunk] = device_activations(device, (chunk,), 0.5, 4000 + k)
     y = torch.empty_like(x)
     tr = {"activations": n}
     for name, mode in (("bsparq", sparq.MODE_BSPARQ), ("vsparq", sparq.MODE_VSPARQ)):
         p = sparq.SparqParams(mode, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
-        ms = time_region(lambda i: sparq.sparq_quantize(x, y, n // 1024, 1024, p), steps, warmup, sync) / steps
+        reps = max(steps, int(np.ceil(MIN_TIMED_MS / (2 * n / (pk["hbm"] * 1e6)))))
+        ms = time_region(lambda i: sparq.sparq_quantize(x, y, n // 1024, 1024, p), reps, warmup, sync) / reps
         gbs = 2 * n / ms / 1e6
         tr[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1),
                     "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
-                                 "frac": round(gbs / pk["hbm"], 4),
-                                 "traffic": (TRANSFORM_TRAFFIC_PER_2P28 * (n >> 28) if name == "bsparq" and n >= (1 << 28) else None),
+                                 "frac": round(gbs / pk["hbm"], 4), "frac_of_nominal_8000": round(gbs / 8000.0, 4),
+                                 "traffic": (TRAFFIC["transform_per_2p28"] * (n >> 28) if name == "bsparq" and n >= (1 << 28) else None),
                                  "peak_source": pk["source"] + " copy"}}
+    sparq.sparq_check()
     return tr
 
 
@@ -199,12 +338,7 @@ def pack_section(device, pk, n, steps, warmup):
     import torch
     import paper_2105_11010_b200 as sparq
     sync = torch.cuda.synchronize
-    gen = torch.Generator(device=device).manual_seed(6)
-    z = torch.randn(n, generator=gen, device=device)
-    x = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
-    x[torch.rand(n, generator=gen, device=device) < 0.5] = 0
-    del z
-    x = x.view(-1, 1024)
+    x = device_activations(device, (n // 1024, 1024), 0.5, 6)
     p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
     cb = sparq.sparq_packed_ctrl_bits(p)
     data = torch.empty(n // 2, dtype=torch.uint8, device=device)
@@ -216,10 +350,7 @@ def pack_section(device, pk, n, steps, warmup):
                      ("unpack", lambda i: sparq.sparq_unpack(data, ctrl, p, y))):
         ms = time_region(fn, steps, warmup, sync) / steps
         gbs = nbytes / ms / 1e6
-        out[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1),
-                     "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
-                                  "frac": round(gbs / pk["hbm"], 4), "traffic": None,
-                                  "peak_source": pk["source"] + " copy"}}
+        out[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1), "frac_of_copy": round(gbs / pk["hbm"], 4)}
     sparq.sparq_check()
     return out
 
@@ -241,50 +372,9 @@ def frontend_section(device, pk, n, steps, warmup):
                                ("quantize_u8", lambda i: sparq.sparq_quantize_act_u8(x, mx, out), n * eb + n)):
             ms = time_region(fn, steps, warmup, sync) / steps
             gbs = nbytes / ms / 1e6
-            res[f"{op}_{name}"] = {"ms": round(ms, 4), "gbs": round(gbs, 1),
-                                   "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"],
-                                                "unit": "GB/s", "frac": round(gbs / pk["hbm"], 4), "traffic": None,
-                                                "peak_source": pk["source"] + " copy"}}
+            res[f"{op}_{name}"] = {"ms": round(ms, 4), "gbs": round(gbs, 1), "frac_of_copy": round(gbs / pk["hbm"], 4)}
     sparq.sparq_check()
     return res
-
-
-def layer1x1_section(device, pk, steps, warmup):
-    """The fused GEMM kernel on an output-heavy 1x1 layer of the ResNet-50 stack at batch 64
-    (56x56x64 -> 256: M 200704, K 64, N 256; vSPARQ n = 4, five placements, round; scale + bias +
-    ReLU + requantize).  Bandwidth-side roofline: bytes = input + output + weights."""
-    import torch
-    import paper_2105_11010_b200 as sparq
-    sync = torch.cuda.synchronize
-    nb, hw, c, cout = 64, 56, 64, 256
-    sets = 4                                         # 4 x (12.8 MB in + 51.4 MB out) = 257 MB > L2
-    gen = torch.Generator(device=device).manual_seed(9)
-    xs = []
-    for _ in range(sets):
-        z = torch.randn(nb * hw * hw * c, generator=gen, device=device)
-        v = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
-        v[torch.rand(v.numel(), generator=gen, device=device) < 0.5] = 0
-        xs.append(v.view(nb, hw, hw, c))
-        del z
-    outs = [torch.empty((nb, hw, hw, cout), dtype=torch.uint8, device=device) for _ in range(sets)]
-    wt = torch.from_numpy(synth.weights(9, (cout, 1, 1, c))).to(device)
-    sc = torch.from_numpy(synth.scales(9, cout)).to(device)
-    bi = torch.from_numpy(synth.bias(9, cout)).to(device)
-    inv = synth.inv_out_scale(c, 0.5)
-    p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
-
-    def step(i):
-        sparq.sparq_conv2d_nhwc_s8(xs[i % sets], wt, (1, 1), (0, 0), p, scale=sc, bias=bi, relu=True,
-                                   inv_out_scale=inv, u8_out=outs[i % sets])
-    ms = time_graph(step, steps, warmup, sync) / steps
-    sparq.sparq_check()
-    nbytes = nb * hw * hw * (c + cout) + cout * c
-    gbs = nbytes / ms / 1e6
-    return {"layer": "56x56x64->256 1x1/s1, batch 64", "ms": round(ms, 4),
-            "tops": round(2 * nb * hw * hw * c * cout / ms / 1e9, 1), "gbs": round(gbs, 1),
-            "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
-                         "frac": round(gbs / pk["hbm"], 4), "traffic": LAYER1X1_TRAFFIC_BYTES, "peak_source": pk["source"] + " copy",
-                         "kernel": "sparq_gemm_kernel<256,64,VSPARQ,4,round>", "algorithmic_bytes_per_launch": nbytes}}
 
 
 def sparse24_section(device, pk, steps, warmup):
@@ -297,12 +387,7 @@ def sparse24_section(device, pk, steps, warmup):
     sync = torch.cuda.synchronize
     M, K, N = 100352, 1152, 128
     p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
-    gen = torch.Generator(device=device).manual_seed(8)
-    z = torch.randn(M * K, generator=gen, device=device)
-    A = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
-    A[torch.rand(M * K, generator=gen, device=device) < 0.5] = 0
-    A = A.view(M, K)
-    del z
+    A = device_activations(device, (M, K), 0.5, 8)
     vals, pos = synth.sparse24_weights(8, N, K)
     w = torch.empty((N, 3 * K), dtype=torch.int8, device=device)
     sparq.sparq_sparse24_expand_weights(torch.from_numpy(vals).to(device), torch.from_numpy(pos).to(device), p, w)
@@ -316,80 +401,153 @@ def sparse24_section(device, pk, steps, warmup):
     sparq.sparq_check()
     gbs = 4 * M * K / ms_e / 1e6
     return {"shape": {"M": M, "K": K, "N": N},
-            "expand_activations": {"ms": round(ms_e, 4), "gbs": round(gbs, 1),
-                                   "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
-                                                "frac": round(gbs / pk["hbm"], 4), "traffic": None,
-                                                "peak_source": pk["source"] + " copy"}},
+            "expand_activations": {"ms": round(ms_e, 4), "gbs": round(gbs, 1), "frac_of_copy": round(gbs / pk["hbm"], 4)},
             "gemm_sparse24": {"ms": round(ms_t, 4), "sparse_tops": round(M * N * K / ms_t / 1e9, 1),
                               "dense_equivalent_tops_executed": round(2 * M * N * 3 * K / ms_t / 1e9, 1)}}
 
 
-def extras(device, pk, steps):
-    """Other workloads of the same library, each with its own roofline: the standalone
-    transform on 2^30 activations and the ResNet-50 layer sweep at batch 64."""
+def layer1x1_section(device, pk, steps, warmup):
+    """The fused GEMM kernel on an output-heavy 1x1 layer of the ResNet-50 stack at batch 64
+    (56x56x64 -> 256: M 200704, K 64, N 256; vSPARQ n = 4, five placements, round; scale + bias +
+    ReLU + requantize).  Bandwidth-side roofline: bytes = input + output + weights."""
+    import paper_2105_11010_b200 as sparq
+    L = dict(nb=64, h=56, w=56, c=64, cout=256, r=1, s=1, stride=1, pad=0, zf=0.5, seed=9)
+    layer = ConvLayer(device, L, sets=4)
+    p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+    ms, _, _ = GraphTimer(layer.fused(p), steps, warmup).run()
+    sparq.sparq_check()
+    nbytes = sum(bytes_of(L))
+    gbs = nbytes / ms / 1e6
+    return {"layer": "56x56x64->256 1x1/s1, batch 64", "ms": round(ms, 4), "tops": round(ops_of(L) / ms / 1e9, 1),
+            "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s",
+                         "frac": round(gbs / pk["hbm"], 4), "traffic": TRAFFIC["layer1x1"],
+                         "peak_source": pk["source"] + " copy", "kernel": "sparq_gemm_kernel (fused 1x1 layer)",
+                         "algorithmic_bytes_per_launch": nbytes}}
+
+
+def cfg1_section(device, steps=200, warmup=10):
+    """Tiny GEMM of config 1 (256 x 576 x 64, 50 % zeros, vSPARQ n = 4 5opt +R; int32 and fp32
+    outputs): microseconds per launch in a back-to-back stream.  Launch-latency bound."""
     import torch
     import paper_2105_11010_b200 as sparq
+    A = torch.from_numpy(synth.activations(0, (256, 576), 0.5)).to(device)
+    B = torch.from_numpy(np.ascontiguousarray(synth.weights(0, (576, 64)).T)).to(device)
+    sc = torch.from_numpy(synth.scales(0, 64)).to(device)
+    acc = torch.empty((256, 64), dtype=torch.int32, device=device)
+    f32 = torch.empty((256, 64), dtype=torch.float32, device=device)
     out = {}
-    sync = torch.cuda.synchronize
-    out["transform_2p30"] = transform_section(device, pk, 1 << 30, 20, 3)
-    out["packed_stream_2p28"] = pack_section(device, pk, 1 << 28, 20, 3)
-    out["minmax_frontend_2p28"] = frontend_section(device, pk, 1 << 28, 20, 3)
-    out["sparse24_vsparq"] = sparse24_section(device, pk, 20, 3)
-    out["gemm_layer1x1"] = layer1x1_section(device, pk, 20, 3)
-    # --- ResNet-50 sweep, batch 64, every conv shape (22 shapes, 52 instances) ---
-    p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
-    layers, total_ms, total_ops = [], 0.0, 0
-    for li, L in enumerate(synth.resnet50_conv_layers()):
-        zf = float(np.random.default_rng(100 + li).uniform(0.3, 0.7))
-        ho, wo = L.out_hw()
-        in_b = 64 * L.h * L.w * L.cin
-        sets = max(2, min(8, int(1.2 * L2_BYTES // (in_b + 64 * ho * wo * L.cout)) + 1))
-        g = torch.Generator(device=device).manual_seed(100 + li)
-        xs = []
-        for _ in range(sets):
-            z = torch.randn(in_b, generator=g, device=device)
-            v = torch.clamp(torch.round(z.abs() * 40.0), 1, 255).to(torch.uint8)
-            v[torch.rand(in_b, generator=g, device=device) < zf] = 0
-            xs.append(v.view(64, L.h, L.w, L.cin))
-        os_ = [torch.empty((64, ho, wo, L.cout), dtype=torch.uint8, device=device) for _ in range(sets)]
-        wt = torch.from_numpy(synth.weights(100 + li, (L.cout, L.r, L.s, L.cin))).to(device)
-        sc = torch.from_numpy(synth.scales(100 + li, L.cout)).to(device)
-        bi = torch.from_numpy(synth.bias(100 + li, L.cout)).to(device)
-        inv = synth.inv_out_scale(L.r * L.s * L.cin, zf)
-
-        def step(i, xs=xs, os_=os_, wt=wt, sc=sc, bi=bi, inv=inv, L=L):
-            sparq.sparq_conv2d_nhwc_s8(xs[i % len(xs)], wt, (L.stride, L.stride), (L.pad, L.pad), p,
-                                       scale=sc, bias=bi, relu=True, inv_out_scale=inv, u8_out=os_[i % len(xs)])
-        ms = time_graph(step, steps, 3, sync) / steps
-        ops = L.ops(64)
-        layers.append({"layer": f"{L.h}x{L.w}x{L.cin}->{L.cout} {L.r}x{L.s}/s{L.stride}", "count": L.count,
-                       "ms": round(ms, 4), "tops": round(ops / ms / 1e9, 1)})
-        total_ms += ms * L.count
-        total_ops += ops * L.count
-        del xs, os_
+    for name, mode in (("vsparq", sparq.MODE_VSPARQ), ("none", sparq.MODE_NONE)):
+        p = sparq.SparqParams(mode, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+        ms, _, _ = GraphTimer(lambda i: sparq.sparq_gemm_s8(A, B, p, scale=sc, acc_out=acc, f32_out=f32), steps, warmup).run(20.0)
+        out[name + "_us"] = round(ms * 1e3, 2)
     sparq.sparq_check()
-    tops = total_ops / total_ms / 1e9
-    int8_peak = pk["bf16"] * INT8_OVER_BF16
-    out["resnet50_sweep_b64"] = {"ms_per_pass": round(total_ms, 3), "tops": round(tops, 1),
-                                 "frac_of_int8_peak": round(tops / int8_peak, 4), "layers": layers}
     return out
 
 
-def cpu_baseline(images: int, repeats: int = 1):
-    """The oracle as it stands on the host cores: `repeats` passes over `images` images of
-    the same layer (transform, direct convolution, epilogue)."""
+def cfg5_section(device, steps=20, warmup=3, full=True):
+    """Ablation grid on the 128 x 28 x 28 x 128 -> 128 3x3 layer: microseconds per step, fused
+    (transform inside the convolution kernel) / unfused (transform kernel into a scratch tensor,
+    then the plain convolution), for the window widths, placement sets and roundings at 50 %
+    zeros, and for the zero fractions with n = 4, five placements, round.  Restricted sets for
+    n = 3 and n = 2 are this library's extension, not the paper's."""
+    import paper_2105_11010_b200 as sparq
+    V, B_ = sparq.MODE_VSPARQ, sparq.MODE_BSPARQ
+    grid = [("v4_5opt_R", V, 4, 0x1F, 1), ("v4_5opt_T", V, 4, 0x1F, 0), ("v4_3opt_R", V, 4, 0x15, 1),
+            ("v4_2opt_R", V, 4, 0x11, 1), ("b4_5opt_R", B_, 4, 0x1F, 1), ("b4_5opt_T", B_, 4, 0x1F, 0),
+            ("v3_6opt_R", V, 3, 0x3F, 1), ("v3_6opt_T", V, 3, 0x3F, 0), ("v3_x35_R", V, 3, 0x35, 1),
+            ("v3_x29_R", V, 3, 0x29, 1), ("v2_7opt_R", V, 2, 0x7F, 1), ("v2_7opt_T", V, 2, 0x7F, 0),
+            ("v2_x55_R", V, 2, 0x55, 1)]
+    if not full:
+        grid = grid[:1] + grid[6:7] + grid[10:11]
+    out = {"us_fused_unfused": {}, "zero_frac_v4_5opt_R": {}}
+    layer = ConvLayer(device, HEAD)
+    for name, mode, n, mask, rnd in grid:
+        p = sparq.SparqParams(mode, n, mask, rnd)
+        f, _, _ = GraphTimer(layer.fused(p), steps, warmup).run()
+        u, _, _ = GraphTimer(layer.unfused(p), steps, warmup).run()
+        out["us_fused_unfused"][name] = [round(f * 1e3, 2), round(u * 1e3, 2)]
+    none, _, _ = GraphTimer(layer.fused(sparq.SparqParams(sparq.MODE_NONE)), steps, warmup).run()
+    out["none_us"] = round(none * 1e3, 2)
+    del layer
+    p = sparq.SparqParams(V, 4, 0x1F, 1)
+    for zf in (0.0, 0.25, 0.5, 0.75, 0.9):
+        L = dict(HEAD, zf=zf, seed=520 + int(zf * 100))
+        layer = ConvLayer(device, L)
+        f, _, _ = GraphTimer(layer.fused(p), steps, warmup).run()
+        u, _, _ = GraphTimer(layer.unfused(p), steps, warmup).run()
+        out["zero_frac_v4_5opt_R"][str(zf)] = [round(f * 1e3, 2), round(u * 1e3, 2)]
+        del layer
+    sparq.sparq_check()
+    return out
+
+
+def sweep_section(device, pk, mma, clk, steps=10, detail=False):
+    """ResNet-50 sweep, batch 64, every conv shape (22 shapes, 52 instances), fused vSPARQ n = 4
+    5opt +R with requantization.  Each layer against its own floor max(ops / tensor peak,
+    bytes / measured copy bandwidth)."""
+    import torch
+    import paper_2105_11010_b200 as sparq
+    p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+    peak_tops = mma["mac_per_clk_sm"] * mma["sms"] * 2 * (clk or 1965.0) * 1e6 / 1e12 if mma else pk["bf16"] * 2
+    layers, total_ms, total_ops, total_floor = [], 0.0, 0, 0.0
+    for li, S in enumerate(synth.resnet50_conv_layers()):
+        zf = float(np.random.default_rng(100 + li).uniform(0.3, 0.7))
+        L = dict(nb=64, h=S.h, w=S.w, c=S.cin, cout=S.cout, r=S.r, s=S.s, stride=S.stride, pad=S.pad, zf=zf, seed=100 + li)
+        layer = ConvLayer(device, L)
+        ms, _, _ = GraphTimer(layer.fused(p), steps, 3).run(25.0)
+        ops, nbytes = ops_of(L), sum(bytes_of(L))
+        floor = max(ops / (peak_tops * 1e12), nbytes / (pk["hbm"] * 1e9)) * 1e3
+        layers.append({"layer": f"{S.h}x{S.w}x{S.cin}->{S.cout} {S.r}x{S.s}/s{S.stride}", "count": S.count,
+                       "us": round(ms * 1e3, 2), "tops": round(ops / ms / 1e9, 1), "floor_us": round(floor * 1e3, 2),
+                       "frac_of_floor": round(floor / ms, 3)})
+        total_ms += ms * S.count
+        total_ops += ops * S.count
+        total_floor += floor * S.count
+        del layer
+        torch.cuda.empty_cache()
+    sparq.sparq_check()
+    tops = total_ops / total_ms / 1e9
+    worst = sorted(layers, key=lambda d: d["frac_of_floor"])[:3]
+    out = {"ms_per_pass": round(total_ms, 4), "tops": round(tops, 1), "frac_of_int8_peak": round(tops / peak_tops, 4),
+           "floor_ms_per_pass": round(total_floor, 4),
+           "worst3": [{k: d[k] for k in ("layer", "us", "floor_us")} for d in worst]}
+    if detail:
+        out["layers"] = layers
+    return out
+
+
+def head_cpu_baseline(budget_s: float = 10.0):
+    """The oracle as it stands on the host cores: whole passes over the full 128-image batch of
+    the headline layer (transform, direct convolution, epilogue) until `budget_s` has gone by."""
     import oracle
-    x = synth.activations(SEED, (images, H, W, C), ZERO_FRAC, stream=10)
-    wt = synth.weights(SEED, (COUT, R, S, C))
-    scale, bias = synth.scales(SEED, COUT), synth.bias(SEED, COUT)
-    inv = synth.inv_out_scale(R * S * C, ZERO_FRAC)
+    L = HEAD
+    x = synth.activations(L["seed"], (L["nb"], L["h"], L["w"], L["c"]), L["zf"], stream=10)
+    wt = synth.weights(L["seed"], (L["cout"], L["r"], L["s"], L["c"]))
+    scale, bias = synth.scales(L["seed"], L["cout"]), synth.bias(L["seed"], L["cout"])
+    inv = synth.inv_out_scale(L["r"] * L["s"] * L["c"], L["zf"])
+    passes = 0
     t0 = time.perf_counter()
-    for _ in range(repeats):
-        acc = oracle.conv2d_nhwc(x, wt, (STRIDE, STRIDE), (PAD, PAD), oracle.MODE_VSPARQ, 4, 0x1F, 1)
+    while True:
+        acc = oracle.conv2d_nhwc(x, wt, (1, 1), (1, 1), oracle.MODE_VSPARQ, 4, 0x1F, 1)
         oracle.epilogue(acc, scale, bias, True, inv)
-    dt = time.perf_counter() - t0
-    ops = 2 * repeats * images * H * W * COUT * R * S * C
-    return ops / dt / 1e12, dt, oracle.num_threads()
+        passes += 1
+        dt = time.perf_counter() - t0
+        if dt >= budget_s or passes >= 64:
+            break
+    return passes * ops_of(L) / dt / 1e12, dt, passes, oracle.num_threads()
+
+
+def reference_step(images: int):
+    import oracle
+    L = HEAD
+    x = synth.activations(L["seed"], (images, L["h"], L["w"], L["c"]), L["zf"], stream=10)
+    wt = synth.weights(L["seed"], (L["cout"], L["r"], L["s"], L["c"]))
+    scale, bias = synth.scales(L["seed"], L["cout"]), synth.bias(L["seed"], L["cout"])
+    inv = synth.inv_out_scale(L["r"] * L["s"] * L["c"], L["zf"])
+    t0 = time.perf_counter()
+    acc = oracle.conv2d_nhwc(x, wt, (1, 1), (1, 1), oracle.MODE_VSPARQ, 4, 0x1F, 1)
+    oracle.epilogue(acc, scale, bias, True, inv)
+    return time.perf_counter() - t0, oracle.num_threads()
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
@@ -407,28 +565,28 @@ def max_over_ranks(ms: float, world: int, device=None) -> float:
 
 def whole_job_tops(ms_per_step: float, world: int) -> float:
     """Weak scaling: each of the `world` replicas does one full workload per step."""
-    return world * OPS_PER_STEP / (ms_per_step * 1e-3) / 1e12
+    return world * ops_of(HEAD) / (ms_per_step * 1e-3) / 1e12
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    images = 2
+    images = 8
     for _ in range(args.warmup):
-        cpu_baseline(images)
-    t0 = time.perf_counter()
-    cores = 1
+        reference_step(images)
+    total, cores = 0.0, 1
     for _ in range(args.steps):
-        _, _, cores = cpu_baseline(images)
-    dt = time.perf_counter() - t0
-    value = args.steps * 2 * images * H * W * COUT * R * S * C / dt / 1e12
-    sample = f"{images} of {NB} images per step"
+        dt, cores = reference_step(images)
+        total += dt
+    ops = 2 * images * HEAD["h"] * HEAD["w"] * HEAD["cout"] * 9 * HEAD["c"]
+    value = args.steps * ops / total / 1e12
+    sample = f"{images} of {HEAD['nb']} images per step"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": "resnet18_conv3x3_b32_56x56x64_to_64 (CPU oracle, " + sample + ")"},
+        "config": {"workload": "ablation_conv3x3_b128_28x28x128_to_128_s1_p1 (CPU oracle, " + sample + ")"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -436,21 +594,23 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+SECTIONS = ["main", "transform", "pack", "frontend", "sparse24", "layer1x1", "mma_peak", "cfg1", "cfg2", "cfg5", "sweep"]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-extras", action="store_true", help="skip the transform and ResNet-50 sweep sections")
-    ap.add_argument("--section", default="main", choices=["main", "transform", "pack", "frontend", "sparse24", "layer1x1"],
-                    help="'transform' times only the standalone transform kernel (small, for profiling)")
-    ap.add_argument("--log2n", type=int, default=28, help="activations for --section transform (2^log2n)")
+    ap.add_argument("--no-extras", action="store_true", help="headline only")
+    ap.add_argument("--full", action="store_true", help="also the codec, front-end and 2:4 sections, and per-layer sweep detail")
+    ap.add_argument("--section", default="main", choices=SECTIONS,
+                    help="print one section in full instead of the headline line (small runs for profiling)")
+    ap.add_argument("--log2n", type=int, default=28, help="activations for the streaming sections (2^log2n)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
-        if args.steps == 400:
-            args.steps = 20
         run_reference(args)
         return
 
@@ -472,83 +632,66 @@ def main():
         if world > 1:
             dist.barrier()
 
-    def sync():
-        torch.cuda.synchronize()
-
+    sync = torch.cuda.synchronize
     pk = peaks()
-    if args.section == "transform":
-        print(json.dumps(transform_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
+    VS = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
+    if args.section != "main":
+        sec = args.section
+        if sec == "transform":
+            res = transform_section(device, pk, 1 << args.log2n, args.steps, args.warmup)
+        elif sec == "pack":
+            res = pack_section(device, pk, 1 << args.log2n, args.steps, args.warmup)
+        elif sec == "frontend":
+            res = frontend_section(device, pk, 1 << args.log2n, args.steps, args.warmup)
+        elif sec == "sparse24":
+            res = sparse24_section(device, pk, args.steps, args.warmup)
+        elif sec == "layer1x1":
+            res = layer1x1_section(device, pk, args.steps, args.warmup)
+        elif sec == "mma_peak":
+            res = mma_peak_section(device)
+        elif sec == "cfg1":
+            res = cfg1_section(device)
+        elif sec == "cfg5":
+            res = cfg5_section(device, args.steps, args.warmup)
+        elif sec == "sweep":
+            res = sweep_section(device, pk, mma_peak_section(device), None, args.steps, detail=True)
+        else:   # cfg2
+            layer = ConvLayer(device, RN18, sets=20, host_recipe=True)
+            ms, _, _ = GraphTimer(layer.fused(VS), args.steps, args.warmup).run()
+            sparq.sparq_check()
+            res = {"us": round(ms * 1e3, 2), "tops": round(ops_of(RN18) / ms / 1e9, 1)}
+        print(json.dumps(res))
         return
-    if args.section == "sparse24":
-        print(json.dumps(sparse24_section(device, pk, args.steps, args.warmup)))
-        return
-    if args.section == "frontend":
-        print(json.dumps(frontend_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
-        return
-    if args.section == "pack":
-        print(json.dumps(pack_section(device, pk, 1 << args.log2n, args.steps, args.warmup)))
-        return
-    if args.section == "layer1x1":
-        print(json.dumps(layer1x1_section(device, pk, args.steps, args.warmup)))
-        return
-    sets = 20   # 20 x (6.4 MB in + 6.4 MB out) = 257 MB > 126 MB of L2
-    xs, outs, wt, scale, bias = build_layer(device, sets)
-    inv = synth.inv_out_scale(R * S * C, ZERO_FRAC)
-    params = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
 
-    def step(i):
-        j = i % sets
-        sparq.sparq_conv2d_nhwc_s8(xs[j], wt, (STRIDE, STRIDE), (PAD, PAD), params, scale=scale, bias=bias,
-                                   relu=True, inv_out_scale=inv, u8_out=outs[j])
-
-    for i in range(args.warmup):
-        step(i)
-    sync()
+    mma = mma_peak_section(device)
+    layer = ConvLayer(device, HEAD, host_recipe=True)
+    step = layer.fused(VS)
+    timer = GraphTimer(step, args.steps, args.warmup)
     sparq.sparq_check()
-    # The K timed steps are captured once into a CUDA graph and replayed, so that the
-    # device-side number is not limited by how fast Python can enqueue ~10 us launches.
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph):
-        for i in range(args.steps):
-            step(args.warmup + i)
     sampler = ClockSampler(local)
-    sync(); barrier()
     sampler.start()
-    # one untimed replay: the first replay of a graph also uploads it to the device
-    graph.replay()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sync(); barrier()
-    e0.record()
-    graph.replay()
-    e1.record()
-    sync(); barrier()
-    ms_total = e0.elapsed_time(e1)
-    # the same K steps enqueued one by one from Python (launch-bound on small layers)
-    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    g0.record()
-    for i in range(args.steps):
-        step(args.warmup + i)
-    g1.record()
-    sync()
-    eager_ms_step = g0.elapsed_time(g1) / args.steps
-    # keep the GPU busy a little longer so that the clock sampler sees it under load
-    t_end = time.time() + 0.6
+    ms_step, timed_ms, replays = timer.run(MIN_TIMED_MS, barrier)
+    # keep the same load running a little longer so that the 50 ms sampler has samples under it
+    t_end = time.time() + 0.4
     while time.time() < t_end:
-        graph.replay()
+        timer.graph.replay()
         sync()
     clocks = sampler.stop()
+    # the same K steps enqueued one by one from Python (launch-bound on small layers)
+    eager_ms_step = time_region(step, args.steps, 0, sync) / args.steps
     sparq.sparq_check()
-    ms_total = max_over_ranks(ms_total, world, device)
-    ms_step = ms_total / args.steps
+    ms_step = max_over_ranks(ms_step, world, device)
     value = whole_job_tops(ms_step, world)
 
     # end to end: pinned host input -> device -> fused kernel -> uint8 result back on the host
-    x_host = torch.from_numpy(synth.activations(SEED, (NB, H, W, C), ZERO_FRAC, stream=10)).pin_memory()
-    y_host = torch.empty((NB, H, W, COUT), dtype=torch.uint8).pin_memory()
+    L = HEAD
+    in_b, out_b, w_b = bytes_of(L)
+    x_host = torch.from_numpy(synth.activations(L["seed"], (L["nb"], L["h"], L["w"], L["c"]), L["zf"], stream=10)).pin_memory()
+    y_host = torch.empty((L["nb"], L["h"], L["w"], L["cout"]), dtype=torch.uint8).pin_memory()
 
     def e2e_step():
-        sparq.sparq_conv2d_nhwc_s8_host(x_host, wt, (STRIDE, STRIDE), (PAD, PAD), params, scale=scale, bias=bias,
-                                        relu=True, inv_out_scale=inv, u8_out=y_host)
+        sparq.sparq_conv2d_nhwc_s8_host(x_host, layer.wt, (1, 1), (1, 1), VS, scale=layer.scale, bias=layer.bias,
+                                        relu=True, inv_out_scale=layer.inv, u8_out=y_host)
     e2e_steps = max(10, min(args.steps, 100))
     for _ in range(3):
         e2e_step()
@@ -559,50 +702,56 @@ def main():
         e2e_step()
     f1.record()
     sync(); barrier()
-    e2e_ms = f0.elapsed_time(f1)
-    e2e_ms = max_over_ranks(e2e_ms, world, device)
+    e2e_ms = max_over_ranks(f0.elapsed_time(f1), world, device)
     e2e_value = whole_job_tops(e2e_ms / e2e_steps, world)
 
-    int8_peak = pk["bf16"] * INT8_OVER_BF16
-    per_launch_tops = OPS_PER_STEP / (ms_step * 1e-3) / 1e12
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 6), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {
-            "workload": "resnet18_conv3x3_b32_56x56x64_to_64_s1_p1 (vSPARQ n=4 5opt +R, scale+bias+ReLU+requant u8)",
-            "global_batch": NB * world, "zero_frac": ZERO_FRAC,
-            "l2": f"rotating {sets} input/output sets ({sets * (IN_BYTES + OUT_BYTES) >> 20} MiB) larger than the 126 MiB L2",
+            "workload": "ablation_conv3x3_b128_28x28x128_to_128_s1_p1, fused vSPARQ n=4 5opt +R, 50% zeros, scale+bias+ReLU+requant u8",
+            "global_batch": L["nb"] * world,
+            "l2": f"rotating {layer.sets} input/output sets ({layer.sets * (in_b + out_b) >> 20} MiB) larger than the 126 MiB L2",
             "parallelism": f"replicas x{world}, batch sharded, no collective",
-            "launch": "K steps captured in one CUDA graph and replayed; eager_ms_per_step is the same loop enqueued from Python",
-            "eager_ms_per_step": eager_ms_step,
+            "timing": f"K steps in one CUDA graph; median of {replays} replays covering {timed_ms:.0f} ms of device time",
+            "eager_ms_per_step": round(eager_ms_step, 5),
         },
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"]},
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": IN_BYTES, "d2h_bytes_per_step": OUT_BYTES,
+        "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": in_b, "d2h_bytes_per_step": out_b,
                 "steps": e2e_steps},
-        "gpu_launches": args.steps,
-        "roofline": {
-            "bound": "tensor", "achieved": per_launch_tops, "peak": int8_peak, "unit": "TOP/s",
-            "frac": per_launch_tops / int8_peak,
-            # dram__bytes_read.sum + dram__bytes_write.sum of one launch (profiles/
-            # sparq_conv_window_kernel_cfg2.txt): the input is read once; the 6.4 MB of
-            # output is still dirty in the 126 MB L2 when the launch ends
-            "traffic": CONV_TRAFFIC_BYTES,
-            "kernel": "sparq_conv_window_kernel<64,64,VSPARQ,4,round,resident> (window implicit-GEMM conv)",
-            "peak_source": f"{pk['source']} bf16 burst {pk['bf16']} TFLOP/s x {INT8_OVER_BF16} (nominal int8:bf16 ratio)",
-            "algorithmic_ops_per_launch": OPS_PER_STEP,
-            "algorithmic_bytes_per_launch": IN_BYTES + OUT_BYTES + WGT_BYTES,
-            "hbm_floor_ms": (IN_BYTES + OUT_BYTES + WGT_BYTES) / (pk["hbm"] * 1e9) * 1e3,
-        },
+        "gpu_launches": args.steps * replays,
+        "roofline": roofline_tensor(ops_of(L), ms_step, mma, pk, clocks["sm_mhz"], TRAFFIC["head"],
+                                    "sparq_conv_window_kernel<128,128,VSPARQ,4,round,resident>", in_b + out_b + w_b),
     }
     if rank == 0 and world == 1:
-        tops, dt, cores = cpu_baseline(NB, repeats=8)
-        line["cpu_baseline"] = {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": f"8 passes over the full {NB}-image batch of the same layer, {dt:.2f} s wall"}
+        tops, dt, passes, cores = head_cpu_baseline()
+        line["cpu_baseline"] = {"value": round(tops, 5), "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{passes} passes over the full {L['nb']}-image batch of the same layer, {dt:.1f} s"}
         if not args.no_extras:
-            del xs, outs
+            del layer, timer
             torch.cuda.empty_cache()
-            line["extra"] = extras(device, pk, 10)
+            ex = {"mma_peak": {k: mma[k] for k in ("mac_per_clk_sm", "sms", "implied_mhz")}}
+            ex["mma_peak"].update({k: mma[k]["mac_per_clk_sm"] for k in ("n64", "n128", "n256")})
+            ex["cfg1_gemm_256x576x64"] = cfg1_section(device)
+            rn = ConvLayer(device, RN18, sets=20, host_recipe=True)
+            ms2, _, _ = GraphTimer(rn.fused(VS), args.steps, 3).run()
+            r2 = roofline_tensor(ops_of(RN18), ms2, mma, pk, clocks["sm_mhz"], TRAFFIC["rn18"], "", sum(bytes_of(RN18)))
+            ex["cfg2_resnet18_conv"] = {"us": round(ms2 * 1e3, 2), "tops": r2["achieved"], "frac": r2["frac"]}
+            del rn
+            torch.cuda.empty_cache()
+            ex["cfg3_resnet50_b64"] = sweep_section(device, pk, mma, clocks["sm_mhz"], 10, detail=args.full)
+            tr = transform_section(device, pk, 1 << 30, 20, 3)
+            ex["cfg4_transform_2p30"] = {m: {"ms": tr[m]["ms"], "gbs": tr[m]["gbs"], "frac_of_copy": tr[m]["roofline"]["frac"],
+                                             "frac_of_8000": tr[m]["roofline"]["frac_of_nominal_8000"]} for m in ("bsparq", "vsparq")}
+            ex["cfg4_transform_2p30"]["traffic"] = tr["bsparq"]["roofline"]["traffic"]
+            ex["cfg5_ablation"] = cfg5_section(device, 20, 3, full=True)
+            if args.full:
+                ex["packed_stream_2p28"] = pack_section(device, pk, 1 << 28, 20, 3)
+                ex["minmax_frontend_2p28"] = frontend_section(device, pk, 1 << 28, 20, 3)
+                ex["sparse24_vsparq"] = sparse24_section(device, pk, 20, 3)
+                ex["gemm_layer1x1"] = layer1x1_section(device, pk, 20, 3)
+            line["extra"] = ex
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
