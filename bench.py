@@ -150,11 +150,16 @@ class GraphTimer:
     def __init__(self, fn, steps, warmup):
         import torch
         self.steps = steps
-        for i in range(warmup):
-            fn(i)
+        # warm-up on the stream the capture will use: the library sets up per-stream state
+        # (workspaces) on a stream's first call, which must not happen inside a capture
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(warmup):
+                fn(i)
         torch.cuda.synchronize()
         self.graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(self.graph):
+        with torch.cuda.graph(self.graph, stream=side):
             for i in range(steps):
                 fn(warmup + i)
         self.graph.replay()            # the first replay also uploads the graph

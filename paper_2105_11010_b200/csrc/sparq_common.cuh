@@ -62,7 +62,38 @@ struct XformDev {
     uint32_t widen_c;
     int rounds;
     int n;
+    // Full placement sets only (every shift 0..8-n allowed; see xform_word_fullset): per 16-bit
+    // half, twice in a word -- the rounding increment, the mask of the kept bits and the
+    // saturation value of the n-bit window (f_*) and of the 2n-bit window of a lone non-zero (l_*).
+    uint32_t f_add, f_mask, f_sat;
+    uint32_t l_add, l_mask, l_sat;
 };
+
+// binary16 bit pattern of an integer 0 < v < 2048 (exact)
+inline uint32_t half_bits_of_int(uint32_t v)
+{
+    int p = 0;
+    while ((v >> (p + 1)) != 0) ++p;
+    return ((uint32_t)(p + 15) << 10) | ((v << (10 - p)) & 0x3FFu);
+}
+
+// Constants of xform_word_fullset for window width n and the rounding flag.
+inline void fill_fullset(XformDev *d, int n, int rnd)
+{
+    auto set = [&](int w, uint32_t *add, uint32_t *mask, uint32_t *sat) {
+        if (w >= 8) {                    // the window holds all 8 bits: nothing is dropped
+            *add = 0u; *mask = 0xFFFFFFFFu; *sat = half_bits_of_int(255u) * 0x00010001u;
+            return;
+        }
+        const uint32_t m16 = (0xFFFFu << (11 - w)) & 0xFFFFu;      // sign, exponent and the top w-1 fraction bits
+        const uint32_t a16 = rnd ? (1u << (10 - w)) : 0u;          // half of the lowest kept bit
+        *mask = m16 * 0x00010001u;
+        *add = a16 * 0x00010001u;
+        *sat = half_bits_of_int(((1u << w) - 1u) << (8 - w)) * 0x00010001u;
+    };
+    set(n, &d->f_add, &d->f_mask, &d->f_sat);
+    set(2 * n, &d->l_add, &d->l_mask, &d->l_sat);
+}
 
 // Mask of the bits BELOW the window for each of the four bytes of x (Section 3.1: the
 // window's top bit is the leading one, or the window sits at the bottom).  The window
@@ -128,5 +159,77 @@ SPARQ_HD uint32_t xform_word(uint32_t x, const XformDev &d)
     uint32_t partner_nz = prmt(nz, nz, 0xAB89u);           // swap within pairs, replicate bit 7
     return (q & partner_nz) | (lone & ~partner_nz);
 }
+
+#ifdef __CUDACC__
+// ---- full placement sets: the window through the floating-point unit --------------------------
+// With every shift allowed, bSPARQ keeps the n most significant bits starting at the leading
+// one (Section 3.1) -- which is what a binary floating-point number with n - 1 fraction bits
+// holds.  A byte b is exact in binary16 (11 significant bits); as bit patterns, two bytes per
+// 32-bit register:
+//     0x6400 | b            = 1024 + b          (one byte permute per pair)
+//     (1024 + b) - 1024     = b, normalized: the subtraction finds the leading one
+//     (bits + half) & mask  = b rounded to n significant bits, ties up, a carry moving into the
+//                             exponent (31 -> 32); without the increment: trimmed
+//     min(., top window)    = the saturation at the top of the byte range (248.. -> 240)
+//     . + 1024              = the integer back in the low byte of each half
+// 13 instructions per four activations for any width and either rounding (17 with the pair
+// rule for n = 4, 26 for n < 4 with its second, 2n-bit window), where the packed integer form
+// with a run-time width needs about twice as many; for n = 4 the integer form specialized at
+// compile time (19 with the pair rule) measured a few per cent faster and is kept.
+__device__ __forceinline__ uint32_t h2_sub(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t h2_add(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("add.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t h2_min(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("min.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+template <int MODE>
+__device__ __forceinline__ uint32_t xform_word_fullset(uint32_t x, const XformDev &d)
+{
+    if (MODE == SPARQ_MODE_NONE) return x;
+    const uint32_t k1024 = 0x64006400u;
+    // bytes 0,1 and bytes 2,3 as halves
+    const uint32_t lo = h2_sub(prmt(x, 0x64646464u, 0x4140u), k1024);
+    const uint32_t hi = h2_sub(prmt(x, 0x64646464u, 0x4342u), k1024);
+    const uint32_t qlo = h2_add(h2_min((lo + d.f_add) & d.f_mask, d.f_sat), k1024);
+    const uint32_t qhi = h2_add(h2_min((hi + d.f_add) & d.f_mask, d.f_sat), k1024);
+    const uint32_t q = prmt(qlo, qhi, 0x6420u);
+    if (MODE == SPARQ_MODE_BSPARQ) return q;
+    // vSPARQ: a byte whose partner is zero keeps the 2n-bit window (the whole byte for n = 4)
+    uint32_t lone = x;
+    if (d.l_mask != 0xFFFFFFFFu) {       // uniform: a kernel argument
+        const uint32_t llo = h2_add(h2_min((lo + d.l_add) & d.l_mask, d.l_sat), k1024);
+        const uint32_t lhi = h2_add(h2_min((hi + d.l_add) & d.l_mask, d.l_sat), k1024);
+        lone = prmt(llo, lhi, 0x6420u);
+    }
+    const uint32_t nz = ((x & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | x;   // bit 7 of each byte: byte != 0
+    const uint32_t partner_nz = prmt(nz, nz, 0xAB89u);           // swap within pairs, replicate bit 7
+    return (q & partner_nz) | (lone & ~partner_nz);
+}
+
+// The transform of a fused kernel instantiated for (MODE, XN, RND): XN = 4 is n = 4 with all
+// five placements (packed-integer form, width fixed at compile time), XN = 8 any other full
+// placement set (6opt, 7opt; either rounding, through the constants; RND unused), XN = 0 the
+// general packed-integer form with run-time width and the placement widening.
+template <int MODE, int XN, bool RND>
+__device__ __forceinline__ uint32_t xform_fused(uint32_t x, const XformDev &d)
+{
+    if (XN == 8) return xform_word_fullset<MODE>(x, d);
+    if (XN == 4) return xform_word<MODE, 4, RND, false>(x, d);
+    return xform_word<MODE, 0, RND, true>(x, d);
+}
+#endif
 
 }  // namespace sparq

@@ -219,6 +219,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
     // this CTA's share of the tile sequence: kernel arguments only, so it is worked out (two
     // integer divisions) while the previous kernel may still be running
     GroupWalk walk(g);
+    bool have = walk.next();       // the first group, too
     dep_launch();
     dep_wait();
 
@@ -233,7 +234,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             bool b_issued = false;  // resident weights requested
             long long pw = 0;
             const long long pt0 = SPARQ_PROF_NOW();
-            while (walk.next()) {
+            for (; have; have = walk.next()) {
                 const int b = rb;                 // window buffer of this group and how often it was used before
                 const uint32_t use = ruse;
                 if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_win_empty[b]), (use - 1) & 1, abort_flag, g.status, g.wait_limit));
@@ -346,7 +347,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             const uint32_t plane16 = (uint32_t)g.plane_bytes >> 4;
             const uint32_t tile16 = (uint32_t)(g.TR * g.Wp * CB) >> 4;
             if (B_RESIDENT) SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, g.wait_limit));
-            while (walk.next()) {
+            for (; have; have = walk.next()) {
                 const int b = rb;
                 const uint32_t wph = ruse & 1u;
                 const uint64_t a_grp = win_desc0 + (uint64_t)((uint32_t)b * (win_bytes >> 4));
@@ -511,7 +512,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             epi_stage_scale_bias<kEpi>(g, 0, BN, et, s_scale, s_bias);
             const uint32_t team = (uint32_t)(warp - kFirstEpiWarp) / kTeamWarps;     // team t takes the tiles of parity t (kAcc is even)
             const int cbase = (((warp - kFirstEpiWarp) % kTeamWarps) >> 2) * kTeamCols;
-            while (walk.next()) {
+            for (; have; have = walk.next()) {
                 for (int j = 0; j < (int)walk.cnt; ++j, ++wt) {
                     if ((wt & 1u) != team) continue;
                     const int oh = ((int)walk.tin + j) * g.TR + tr;
@@ -549,7 +550,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 rb[i] = s_bias[cbase + i];
             }
             uint32_t pre_full = 0;     // the next tile's accumulator was seen complete
-            while (walk.next()) {
+            for (; have; have = walk.next()) {
               for (int j = 0; j < (int)walk.cnt; ++j, ++wt) {
                 const uint32_t acc = wt & (uint32_t)(kAcc - 1);
                 // coordinates first: they do not depend on the accumulator
@@ -598,7 +599,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
               }
             }
         } else
-        while (walk.next()) {
+        for (; have; have = walk.next()) {
           for (int j = 0; j < (int)walk.cnt; ++j, ++wt) {
             const int64_t nt = (int64_t)walk.nt;
             const int acc = (int)(wt & (uint32_t)(kAcc - 1));
@@ -631,7 +632,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
         int rb = 0; uint32_t ruse = 0;         // window buffer of the group (gi % win_bufs) and its use count (gi / win_bufs)
         long long xw = 0;
         const long long xt0 = SPARQ_PROF_NOW();
-        while (walk.next()) {
+        for (; have; have = walk.next()) {
             const int b = rb;
             const uint32_t wph = ruse & 1u;
             for (int j = 0; j < g.G; ++j) {
@@ -657,10 +658,10 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 if (!ok[q]) continue;
-                                v[q].x = xform_word<MODE, XN, RND, XN == 0>(v[q].x, xf);
-                                v[q].y = xform_word<MODE, XN, RND, XN == 0>(v[q].y, xf);
-                                v[q].z = xform_word<MODE, XN, RND, XN == 0>(v[q].z, xf);
-                                v[q].w = xform_word<MODE, XN, RND, XN == 0>(v[q].w, xf);
+                                v[q].x = xform_fused<MODE, XN, RND>(v[q].x, xf);
+                                v[q].y = xform_fused<MODE, XN, RND>(v[q].y, xf);
+                                v[q].z = xform_fused<MODE, XN, RND>(v[q].z, xf);
+                                v[q].w = xform_fused<MODE, XN, RND>(v[q].w, xf);
                                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
                                              :: "r"(pbase + (v0 + (uint32_t)q * kXfThreads) * 16u),
                                                 "r"(v[q].x), "r"(v[q].y), "r"(v[q].z), "r"(v[q].w) : "memory");
@@ -723,11 +724,13 @@ cudaError_t launch_window_shape(const CUtensorMap &mx0, const CUtensorMap &mx1, 
         constexpr bool RES = RES_;                                                                     \
         if (mode == SPARQ_MODE_NONE) SPARQ_LAUNCH_WINDOW_VARIANT(SPARQ_MODE_NONE, 4, false);           \
         if (mode == SPARQ_MODE_BSPARQ) {                                                               \
+            if (n == 8) SPARQ_LAUNCH_WINDOW_VARIANT(SPARQ_MODE_BSPARQ, 8, true);                       \
             if (n == 4) { if (rnd) SPARQ_LAUNCH_WINDOW_VARIANT(SPARQ_MODE_BSPARQ, 4, true);            \
                           else SPARQ_LAUNCH_WINDOW_VARIANT(SPARQ_MODE_BSPARQ, 4, false); }             \
             if (rnd) SPARQ_LAUNCH_WINDOW_VARIANT(SPARQ_MODE_BSPARQ, 0, true);                          \
             else SPARQ_LAUNCH_WINDOW_VARIANT(SPARQ_MODE_BSPARQ, 0, false);                             \
         }                                                                                              \
+        if (n == 8) SPARQ_LAUNCH_WINDOW_VARIANT(SPARQ_MODE_VSPARQ, 8, true);                           \
         if (n == 4) { if (rnd) SPARQ_LAUNCH_WINDOW_VARIANT(SPARQ_MODE_VSPARQ, 4, true);                \
                       else SPARQ_LAUNCH_WINDOW_VARIANT(SPARQ_MODE_VSPARQ, 4, false); }                 \
         if (rnd) SPARQ_LAUNCH_WINDOW_VARIANT(SPARQ_MODE_VSPARQ, 0, true);                              \

@@ -146,6 +146,7 @@ static int next_transform_args(const sparq_epilogue *e, int64_t N, int *mode, in
     *mode = SPARQ_MODE_NONE;
     *rnd = 0;
     *xf = XformDev{0u, 0, 4};
+    fill_fullset(xf, 4, 0);
     if (!e->next_transform || e->next_transform->mode == SPARQ_MODE_NONE) return SPARQ_OK;
     XformArgs nx;
     int rc = validate_params(e->next_transform, &nx);
@@ -155,6 +156,7 @@ static int next_transform_args(const sparq_epilogue *e, int64_t N, int *mode, in
     *mode = nx.mode;
     *rnd = nx.rnd;
     *xf = XformDev{nx.widen_c, nx.widen_rounds, nx.n};
+    fill_fullset(xf, nx.n, nx.rnd);
     return SPARQ_OK;
 }
 
@@ -207,9 +209,17 @@ static int pick_bn(int64_t M, int64_t N, int sms, bool transform)
     return best;
 }
 
-// Window-width argument of the launchers: 4 selects the kernels specialized for n = 4 with
-// all five placements; anything else (0) the general ones.
-static int variant_n(const XformArgs &x) { return (x.n == 4 && x.widen_rounds == 0) ? 4 : 0; }
+// Variant argument of the launchers: 4 = n = 4 with all five placements, 8 = another full
+// placement set (6opt, 7opt), 0 = the general kernels.
+static int variant_n(const XformArgs &x) { return x.widen_rounds != 0 ? 0 : (x.n == 4 ? 4 : 8); }
+
+// Kernel-side transform constants.
+static XformDev xform_dev(const XformArgs &x)
+{
+    XformDev d{x.widen_c, x.widen_rounds, x.n};
+    fill_fullset(&d, x.n, x.rnd);
+    return d;
+}
 
 static cudaError_t launch(int bn, int bk, const CUtensorMap &ma, const CUtensorMap &mb, const GemmArgs &g,
                           const XformArgs &x, int grid, cudaStream_t st)
@@ -224,7 +234,7 @@ static cudaError_t launch(int bn, int bk, const CUtensorMap &ma, const CUtensorM
 
 static int fill_common(GemmArgs *g, const XformArgs &x, const sparq_epilogue *e, unsigned int *status)
 {
-    g->xf = XformDev{x.widen_c, x.widen_rounds, x.n};
+    g->xf = xform_dev(x);
     g->scale = e->scale;
     g->bias = e->bias;
     g->relu = e->relu ? 1 : 0;
@@ -408,7 +418,7 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     g.plane_bytes = plane_bytes;
     g.win_bufs = win_bufs;
     g.b_stages = b_stages;
-    g.xf = XformDev{x.widen_c, x.widen_rounds, x.n};
+    g.xf = xform_dev(x);
     g.scale = e->scale; g.bias = e->bias; g.relu = e->relu ? 1 : 0; g.inv_out_scale = e->inv_out_scale;
     g.acc_out = e->acc_out; g.f32_out = e->f32_out; g.u8_out = e->u8_out;
     g.status = status;

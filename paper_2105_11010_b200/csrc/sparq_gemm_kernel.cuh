@@ -368,14 +368,16 @@ __device__ __forceinline__ uint32_t pack4(uint32_t a, uint32_t b, uint32_t c, ui
 // instruction caches, which the warp roles share.
 static __device__ __noinline__ void next_xform_words(uint32_t *w, int count, int mode, int rnd, XformDev xf)
 {
-    const bool fast4 = xf.n == 4 && xf.rounds == 0;   // n = 4, all five placements
+    const bool full = xf.rounds == 0 && xf.n != 4;   // 6opt / 7opt: the half-precision form
     for (int q = 0; q < count; ++q) {
         uint32_t x = w[q];
         if (mode == SPARQ_MODE_VSPARQ) {
-            if (fast4) x = rnd ? xform_word<SPARQ_MODE_VSPARQ, 4, true, false>(x, xf) : xform_word<SPARQ_MODE_VSPARQ, 4, false, false>(x, xf);
+            if (full) x = xform_word_fullset<SPARQ_MODE_VSPARQ>(x, xf);
+            else if (xf.rounds == 0) x = rnd ? xform_word<SPARQ_MODE_VSPARQ, 4, true, false>(x, xf) : xform_word<SPARQ_MODE_VSPARQ, 4, false, false>(x, xf);
             else x = rnd ? xform_word<SPARQ_MODE_VSPARQ, 0, true, true>(x, xf) : xform_word<SPARQ_MODE_VSPARQ, 0, false, true>(x, xf);
         } else {
-            if (fast4) x = rnd ? xform_word<SPARQ_MODE_BSPARQ, 4, true, false>(x, xf) : xform_word<SPARQ_MODE_BSPARQ, 4, false, false>(x, xf);
+            if (full) x = xform_word_fullset<SPARQ_MODE_BSPARQ>(x, xf);
+            else if (xf.rounds == 0) x = rnd ? xform_word<SPARQ_MODE_BSPARQ, 4, true, false>(x, xf) : xform_word<SPARQ_MODE_BSPARQ, 4, false, false>(x, xf);
             else x = rnd ? xform_word<SPARQ_MODE_BSPARQ, 0, true, true>(x, xf) : xform_word<SPARQ_MODE_BSPARQ, 0, false, true>(x, xf);
         }
         w[q] = x;
@@ -937,10 +939,10 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                                      : "r"(base + (uint32_t)((j0 + j) * kXfThreads * 16)));
 #pragma unroll
                     for (int j = 0; j < kBatch; ++j) {
-                        v[j].x = xform_word<MODE, XN, RND, XN == 0>(v[j].x, xf);
-                        v[j].y = xform_word<MODE, XN, RND, XN == 0>(v[j].y, xf);
-                        v[j].z = xform_word<MODE, XN, RND, XN == 0>(v[j].z, xf);
-                        v[j].w = xform_word<MODE, XN, RND, XN == 0>(v[j].w, xf);
+                        v[j].x = xform_fused<MODE, XN, RND>(v[j].x, xf);
+                        v[j].y = xform_fused<MODE, XN, RND>(v[j].y, xf);
+                        v[j].z = xform_fused<MODE, XN, RND>(v[j].z, xf);
+                        v[j].w = xform_fused<MODE, XN, RND>(v[j].w, xf);
                         asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
                                      :: "r"(base + (uint32_t)((j0 + j) * kXfThreads * 16)),
                                         "r"(v[j].x), "r"(v[j].y), "r"(v[j].z), "r"(v[j].w) : "memory");
@@ -1015,11 +1017,13 @@ cudaError_t launch_gemm_shape(const CUtensorMap &ma, const CUtensorMap &mb, cons
         constexpr int BN = BN_, BK = BK_;                                                              \
         if (mode == SPARQ_MODE_NONE) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_NONE, 4, false);                  \
         if (mode == SPARQ_MODE_BSPARQ) {                                                               \
+            if (n == 8) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_BSPARQ, 8, true);                              \
             if (n == 4) { if (rnd) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_BSPARQ, 4, true);                   \
                           else SPARQ_LAUNCH_VARIANT(SPARQ_MODE_BSPARQ, 4, false); }                    \
             if (rnd) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_BSPARQ, 0, true);                                 \
             else SPARQ_LAUNCH_VARIANT(SPARQ_MODE_BSPARQ, 0, false);                                    \
         }                                                                                              \
+        if (n == 8) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_VSPARQ, 8, true);                                  \
         if (n == 4) { if (rnd) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_VSPARQ, 4, true);                       \
                       else SPARQ_LAUNCH_VARIANT(SPARQ_MODE_VSPARQ, 4, false); }                        \
         if (rnd) SPARQ_LAUNCH_VARIANT(SPARQ_MODE_VSPARQ, 0, true);                                     \
