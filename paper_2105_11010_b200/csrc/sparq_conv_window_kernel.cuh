@@ -52,6 +52,9 @@ struct WindowArgs {
     int w_one_copy;         // resident weights: map_w is the 3-D (bytes, rows, blocks) view and one copy brings all blocks
     uint32_t n_tiles;       // column tiles
     uint32_t units;         // n_img * tiles_per_img * n_tiles, column tile fastest
+    uint32_t groups;        // streamed weights on 128-wide tiles: n_img * n_tiles * ceil(tiles_per_img / G) whole
+                            // groups of up to G row tiles of one (image, column tile), which share one pass over
+                            // the weights; CTAs own whole groups there, contiguous shares of the unit sequence else
     // transform
     XformDev xf;
     // epilogue
@@ -75,7 +78,7 @@ struct WindowArgs {
 constexpr int kWindowMaxDynSmem = 232448 - 4096;
 constexpr int kMaxWinBufs = 4;
 constexpr int kMaxG = 8;
-constexpr int kMaxBStages = 8;
+constexpr int kMaxBStages = 12;
 // Two warps issue MMAs, taking the tiles of a CTA alternately (each owns one of the two
 // accumulators): whatever one of them does between two tiles -- commits, barrier reads that
 // queue behind the tensor core's own shared-memory traffic, descriptor set-up -- happens
@@ -100,15 +103,17 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
 // Walks the groups of one CTA's share of the tile sequence.  Every warp role runs the same
 // walk, so that window buffers, accumulators and barrier phases line up without any
 // communication.
+template <bool BY_GROUP>
 struct GroupWalk {
-    uint32_t u, u_end;          // units still to do: [u, u_end)
+    uint32_t u, u_end;          // units (BY_GROUP: whole groups) still to do: [u, u_end)
     uint32_t n_tiles, tpi, G;
     uint32_t img, tin, nt, cnt; // current group: image, first tile inside it, column tile, tiles
 
     __device__ __forceinline__ GroupWalk(const WindowArgs &g)
     {
-        // units split into gridDim.x contiguous shares that differ by at most one
-        const uint32_t q = g.units / gridDim.x, rem = g.units - q * gridDim.x;
+        // the sequence is split into gridDim.x contiguous shares that differ by at most one
+        const uint32_t total = BY_GROUP ? g.groups : g.units;
+        const uint32_t q = total / gridDim.x, rem = total - q * gridDim.x;
         u = blockIdx.x * q + (blockIdx.x < rem ? blockIdx.x : rem);
         u_end = u + q + (blockIdx.x < rem ? 1u : 0u);
         n_tiles = g.n_tiles; tpi = (uint32_t)g.tiles_per_img; G = (uint32_t)g.G;
@@ -117,6 +122,17 @@ struct GroupWalk {
     __device__ __forceinline__ bool next()
     {
         if (u >= u_end) return false;
+        if (BY_GROUP) {
+            // group number u = (image * n_tiles + column tile) * gpt + k: tiles k*G .. of that image
+            const uint32_t gpt = (tpi + G - 1) / G;
+            const uint32_t key = u / gpt, k = u - key * gpt;
+            img = key / n_tiles;
+            nt = key - img * n_tiles;
+            tin = k * G;
+            cnt = tpi - tin < G ? tpi - tin : G;
+            u += 1;
+            return true;
+        }
         uint32_t mt = u;
         nt = 0;
         if (n_tiles != 1) { mt = u / n_tiles; nt = u - mt * n_tiles; }
@@ -145,8 +161,12 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
     __shared__ __align__(8) uint64_t bar_win_empty[kMaxWinBufs];
     __shared__ __align__(8) uint64_t bar_b_full[kMaxBStages], bar_b_empty[kMaxBStages];
     // Accumulator stages in tensor memory; tile number t uses stage t % kAcc.  (Four stages were
-    // measured and changed nothing: the epilogue hands a stage back well within one tile.)
-    constexpr int kAcc = 2;
+    // measured and changed nothing for tiles that run one after the other: the epilogue hands a
+    // stage back well within one tile.)  Streamed weights on 128-wide tiles: the tiles of a group
+    // are accumulated TOGETHER during one pass over the weights (kBatched), so a group holds up
+    // to two stages and four let the next group start while the previous one is in its epilogue.
+    constexpr bool kBatched = !B_RESIDENT && BN == 128;
+    constexpr int kAcc = kBatched ? 4 : 2;
     __shared__ __align__(8) uint64_t bar_acc_full[kAcc], bar_acc_empty[kAcc], bar_done;
     __shared__ uint32_t tmem_base_slot;
     __shared__ uint32_t abort_word;
@@ -218,7 +238,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
     const uint32_t tmem_base = tmem_base_slot;
     // this CTA's share of the tile sequence: kernel arguments only, so it is worked out (two
     // integer divisions) while the previous kernel may still be running
-    GroupWalk walk(g);
+    GroupWalk<kBatched> walk(g);
     bool have = walk.next();       // the first group, too
     dep_launch();
     dep_wait();
@@ -285,7 +305,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 if (++rb == g.win_bufs) { rb = 0; ++ruse; }
                 if (!B_RESIDENT) {
                     bool stop = false;
-                    for (int j = 0; j < (int)walk.cnt && !stop; ++j) {
+                    const int passes = kBatched ? 1 : (int)walk.cnt;     // batched: one pass serves the whole group
+                    for (int j = 0; j < passes && !stop; ++j) {
                         for (int cb = 0; cb < g.c_blocks && !stop; ++cb) {
                             for (int tap = 0; tap < taps; ++tap, ++it) {
                                 const int s = it % g.b_stages;
@@ -359,6 +380,54 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 // queued; when both say "ready" -- the usual case -- that tile starts without
                 // touching shared memory.
                 uint32_t pre_acc = 0, pre_ops = 0;
+                if constexpr (kBatched) {
+                    // One pass over the streamed weights for all tiles of the group: every weight
+                    // block is fetched from L2 once per group instead of once per tile.  Warp 1
+                    // issues; the other issuer only keeps its counters in step.
+                    const int cnt = (int)walk.cnt;
+                    if (me == 0) {
+                        issued = true;
+                        for (int j = 0; j < cnt; ++j) {
+                            const uint32_t t = wt + (uint32_t)j, use = t / (uint32_t)kAcc;
+                            if (use > 0) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[t & (uint32_t)(kAcc - 1)]), (use - 1) & 1, abort_flag, g.status, g.wait_limit));
+                        }
+                        // all pieces of the group: the transform warps finish them in order; without a
+                        // transform the copies land in any order
+                        if (MODE == SPARQ_MODE_NONE) {
+                            for (int j = 0; j < cnt; ++j)
+                                SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), wph, abort_flag, g.status, g.wait_limit));
+                        } else {
+                            SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b * kMaxG + cnt - 1]), wph, abort_flag, g.status, g.wait_limit));
+                        }
+                        tc_fence_after();
+                        uint64_t a_cb = a_grp;
+                        for (uint32_t cb = 0; cb < (uint32_t)g.c_blocks; ++cb, a_cb += plane16) {
+                            uint64_t a_r = a_cb;
+                            for (int r = 0; r < g.R; ++r, a_r += row16) {
+                                for (int sx = 0; sx < g.S; ++sx) {
+                                    SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status, g.wait_limit));
+                                    tc_fence_after();
+                                    const uint64_t bdesc = b_desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kBBlock >> 4));
+                                    const uint64_t a_tap = a_r + (uint64_t)(uint32_t)(sx * (CB >> 4));
+                                    const uint32_t first = (cb == 0 && r == 0 && sx == 0) ? 0u : 1u;
+                                    for (int j = 0; j < cnt; ++j) {
+                                        const uint32_t d_tmem = tmem_base + ((wt + (uint32_t)j) & (uint32_t)(kAcc - 1)) * (uint32_t)BN;
+                                        const uint64_t adesc = a_tap + (uint64_t)((uint32_t)j * tile16);
+#pragma unroll
+                                        for (int k = 0; k < CB / 32; ++k)
+                                            tc_mma_i8_if(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
+                                                         (first || k > 0) ? 1u : 0u, elected);
+                                    }
+                                    tc_commit_if(smem_u32(&bar_b_empty[s]), elected);
+                                    if (++s == g.b_stages) { s = 0; bph ^= 1u; }
+                                }
+                            }
+                        }
+                        for (int j = 0; j < cnt; ++j)
+                            tc_commit_if(smem_u32(&bar_acc_full[(wt + (uint32_t)j) & (uint32_t)(kAcc - 1)]), elected);
+                    }
+                    wt += (uint32_t)cnt;
+                } else
                 for (int j = 0; j < (int)walk.cnt; ++j, ++wt) {
                     if (g.issuers == 2 ? (wt & 1u) != me : me != 0u) {
                         if (!B_RESIDENT) {

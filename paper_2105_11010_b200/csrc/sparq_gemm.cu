@@ -338,7 +338,7 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     const int n_tiles = (cout + bn - 1) / bn;
     const int64_t units = m_tiles * n_tiles;
     if (units >= (int64_t)1 << 31) return 0;
-    const int grid = (int)(units < sms ? units : sms);
+    int grid = (int)(units < sms ? units : sms);
 
     // Shared memory of one window buffer when up to `grp` tiles share it: a plane (one channel
     // block) holds every row the MMA of the group's last tile may touch.
@@ -356,7 +356,7 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
         if (gmax > kMaxG) gmax = kMaxG;
         if (cb == 64 && (((tr * wp) & 1) || (((r - 1) * wp) & 1))) gmax = 1;
     }
-    bool resident = false;
+    bool resident = false, batched = false;
     int win_bufs = 2, b_stages = 0, grp = 1;
     if (bn != 256 && n_tiles == 1 && 1024 + 2 * plane_for(1) * c_blocks + kb_count * b_block <= kMaxDynSmem) {
         resident = true;
@@ -369,15 +369,23 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
                1024 + (win_bufs + 1) * plane_for(grp) * c_blocks + kb_count * b_block <= kMaxDynSmem) ++win_bufs;
     } else {
         if (bn == 64) return 0;                          // only the resident form is built for 64-wide tiles
-        grp = gmax;
+        // 128-wide tiles: up to two row tiles of one (image, column tile) are accumulated together
+        // during ONE pass over the streamed weights (four accumulator stages: two groups in
+        // flight), which halves the weight traffic out of L2 -- the bound of these layers.
+        batched = bn == 128;
+        grp = batched ? (tiles_per_img < 2 ? tiles_per_img : 2) : gmax;
         while (grp > 1 && kMaxDynSmem - 1024 - 2 * plane_for(grp) * c_blocks < 4 * b_block) --grp;
         const int win_bytes1 = plane_for(grp) * c_blocks;
-        const int left = kMaxDynSmem - 1024 - 2 * win_bytes1;
+        // a CTA that owns a single group needs no second window buffer: the room goes to the
+        // weight ring, whose depth (bytes in flight) bounds how fast one SM can pull the weights
+        const int64_t groups_b = (int64_t)n * n_tiles * ((tiles_per_img + grp - 1) / grp);
+        if (batched && groups_b <= sms) win_bufs = 1;
+        const int left = kMaxDynSmem - 1024 - win_bufs * win_bytes1;
         b_stages = left / b_block;
         if (b_stages > kMaxBStages) b_stages = kMaxBStages;
         if (b_stages < 2) return 0;
         // spare room beyond four weight stages goes to a third window buffer
-        if (b_stages > 4 && 1024 + 3 * win_bytes1 + 4 * b_block <= kMaxDynSmem) {
+        if (win_bufs == 2 && b_stages > 4 && 1024 + 3 * win_bytes1 + 4 * b_block <= kMaxDynSmem) {
             win_bufs = 3;
             b_stages = (kMaxDynSmem - 1024 - 3 * win_bytes1) / b_block;
             if (b_stages > kMaxBStages) b_stages = kMaxBStages;
@@ -415,6 +423,12 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     g.piece_bytes = cb * wp * tr;
     g.n_tiles = (uint32_t)n_tiles;
     g.units = (uint32_t)units;
+    if (batched) {
+        // CTAs own whole groups, so that a group is never cut at a share boundary
+        const int64_t groups = (int64_t)n * n_tiles * ((tiles_per_img + grp - 1) / grp);
+        g.groups = (uint32_t)groups;
+        grid = (int)(groups < sms ? groups : sms);
+    }
     g.plane_bytes = plane_bytes;
     g.win_bufs = win_bufs;
     g.b_stages = b_stages;
