@@ -172,7 +172,7 @@ class GraphTimer:
         probe0.record(); self.graph.replay(); probe1.record()
         torch.cuda.synchronize()
         one = max(probe0.elapsed_time(probe1), 1e-3)
-        n = int(min(2000, max(5, np.ceil(min_ms / one))))
+        n = int(min(2000, max(5, np.ceil(1.2 * min_ms / one))))
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
         torch.cuda.synchronize()
         if barrier:
@@ -268,14 +268,11 @@ def roofline_tensor(ops, ms, mma, pk, clocks_mhz, traffic, kernel, alg_bytes):
     return {
         "bound": "tensor", "achieved": round(tops, 1), "peak": round(peak, 1), "unit": "TOP/s",
         "frac": round(tops / peak, 4), "traffic": traffic,
-        "peak_source": (f"own MMA-only kind::i8 loop: {mma['mac_per_clk_sm']:.0f} MAC/clk/SM x {mma['sms']} SMs x "
+        "peak_source": (f"measured: own MMA-only kind::i8 loop, {mma['mac_per_clk_sm']:.0f} MAC/clk/SM x {mma['sms']} SMs x "
                         f"{clk:.0f} MHz sampled" if mma else f"{pk['source']} bf16 burst x 2"),
-        "frac_of_2x_bf16_burst": round(tops / (pk["bf16"] * 2), 4),
         "frac_of_nominal_4500": round(tops / NOMINAL_INT8_TOPS, 4),
-        "timing": "median CUDA-graph replay / steps: per step in a back-to-back stream (a launch's prologue overlaps "
-                  "its predecessor's tail), not per isolated launch",
-        "kernel": kernel, "algorithmic_ops_per_launch": ops, "algorithmic_bytes_per_launch": alg_bytes,
-        "hbm_floor_ms": round(alg_bytes / (pk["hbm"] * 1e9) * 1e3, 5),
+        "per": "step in a back-to-back stream, not an isolated launch",
+        "kernel": kernel, "ops": ops, "bytes": alg_bytes,
     }
 
 
@@ -464,13 +461,13 @@ def cfg5_section(device, steps=20, warmup=3, full=True):
             ("v2_x55_R", V, 2, 0x55, 1)]
     if not full:
         grid = grid[:1] + grid[6:7] + grid[10:11]
-    out = {"us_fused_unfused": {}, "zero_frac_v4_5opt_R": {}}
+    out = {"us_fused_unfused": {}, "zero_frac_v4_5opt_R": {}}    # microseconds: [fused, unfused]
     layer = ConvLayer(device, HEAD)
     for name, mode, n, mask, rnd in grid:
         p = sparq.SparqParams(mode, n, mask, rnd)
         f, _, _ = GraphTimer(layer.fused(p), steps, warmup).run()
         u, _, _ = GraphTimer(layer.unfused(p), steps, warmup).run()
-        out["us_fused_unfused"][name] = [round(f * 1e3, 2), round(u * 1e3, 2)]
+        out["us_fused_unfused"][name] = [round(f * 1e3, 1), round(u * 1e3, 1)]
     none, _, _ = GraphTimer(layer.fused(sparq.SparqParams(sparq.MODE_NONE)), steps, warmup).run()
     out["none_us"] = round(none * 1e3, 2)
     del layer
@@ -480,7 +477,7 @@ def cfg5_section(device, steps=20, warmup=3, full=True):
         layer = ConvLayer(device, L)
         f, _, _ = GraphTimer(layer.fused(p), steps, warmup).run()
         u, _, _ = GraphTimer(layer.unfused(p), steps, warmup).run()
-        out["zero_frac_v4_5opt_R"][str(zf)] = [round(f * 1e3, 2), round(u * 1e3, 2)]
+        out["zero_frac_v4_5opt_R"][str(zf)] = [round(f * 1e3, 1), round(u * 1e3, 1)]
         del layer
     sparq.sparq_check()
     return out
@@ -515,7 +512,7 @@ def sweep_section(device, pk, mma, clk, steps=10, detail=False):
     worst = sorted(layers, key=lambda d: d["frac_of_floor"])[:3]
     out = {"ms_per_pass": round(total_ms, 4), "tops": round(tops, 1), "frac_of_int8_peak": round(tops / peak_tops, 4),
            "floor_ms_per_pass": round(total_floor, 4),
-           "worst3": [{k: d[k] for k in ("layer", "us", "floor_us")} for d in worst]}
+           "worst3": [[d["layer"], d["us"], d["floor_us"]] for d in worst]}
     if detail:
         out["layers"] = layers
     return out
@@ -715,11 +712,11 @@ def main():
         "warmup": args.warmup, "ms_per_step": round(ms_step, 6), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {
-            "workload": "ablation_conv3x3_b128_28x28x128_to_128_s1_p1, fused vSPARQ n=4 5opt +R, 50% zeros, scale+bias+ReLU+requant u8",
+            "workload": "cfg5 conv3x3 128x28x28x128->128 s1 p1, fused vSPARQ n=4 5opt +R, 50% zeros, requant u8",
             "global_batch": L["nb"] * world,
-            "l2": f"rotating {layer.sets} input/output sets ({layer.sets * (in_b + out_b) >> 20} MiB) larger than the 126 MiB L2",
-            "parallelism": f"replicas x{world}, batch sharded, no collective",
-            "timing": f"K steps in one CUDA graph; median of {replays} replays covering {timed_ms:.0f} ms of device time",
+            "l2": f"{layer.sets} rotating in/out sets, {layer.sets * (in_b + out_b) >> 20} MiB > 126 MiB L2",
+            "parallelism": f"replicas x{world}, no collective",
+            "timing": f"K steps per CUDA graph; median of {replays} replays ({timed_ms:.0f} ms)",
             "eager_ms_per_step": round(eager_ms_step, 5),
         },
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"]},
@@ -732,12 +729,11 @@ def main():
     if rank == 0 and world == 1:
         tops, dt, passes, cores = head_cpu_baseline()
         line["cpu_baseline"] = {"value": round(tops, 5), "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": f"{passes} passes over the full {L['nb']}-image batch of the same layer, {dt:.1f} s"}
+                                "sample": f"{passes} passes over the full {L['nb']}-image batch, {dt:.1f} s"}
         if not args.no_extras:
             del layer, timer
             torch.cuda.empty_cache()
-            ex = {"mma_peak": {k: mma[k] for k in ("mac_per_clk_sm", "sms", "implied_mhz")}}
-            ex["mma_peak"].update({k: mma[k]["mac_per_clk_sm"] for k in ("n64", "n128", "n256")})
+            ex = {"mma_peak_mac_per_clk_sm": {k: mma[k]["mac_per_clk_sm"] for k in ("n64", "n128", "n256")}}
             ex["cfg1_gemm_256x576x64"] = cfg1_section(device)
             rn = ConvLayer(device, RN18, sets=20, host_recipe=True)
             ms2, _, _ = GraphTimer(rn.fused(VS), args.steps, 3).run()
@@ -749,7 +745,7 @@ def main():
             tr = transform_section(device, pk, 1 << 30, 20, 3)
             ex["cfg4_transform_2p30"] = {m: {"ms": tr[m]["ms"], "gbs": tr[m]["gbs"], "frac_of_copy": tr[m]["roofline"]["frac"],
                                              "frac_of_8000": tr[m]["roofline"]["frac_of_nominal_8000"]} for m in ("bsparq", "vsparq")}
-            ex["cfg4_transform_2p30"]["traffic"] = tr["bsparq"]["roofline"]["traffic"]
+            ex["cfg4_transform_2p30"].update(bound="hbm", peak_gbs=pk["hbm"], traffic=tr["bsparq"]["roofline"]["traffic"])
             ex["cfg5_ablation"] = cfg5_section(device, 20, 3, full=True)
             if args.full:
                 ex["packed_stream_2p28"] = pack_section(device, pk, 1 << 28, 20, 3)
