@@ -48,6 +48,7 @@ struct WindowArgs {
     int plane_bytes;        // shared-memory bytes reserved per channel block (>= rows the MMA may touch)
     int win_bufs;           // window buffers in the ring
     int b_stages;           // weight stages (stream mode) or resident blocks (resident mode)
+    int early_weights;      // resident weights may be fetched before the previous kernel on the stream has finished
     int issuers;            // 2: the two issuer warps alternate (resident weights); 1: warp 1 issues every tile (streamed weights)
     int w_one_copy;         // resident weights: map_w is the 3-D (bytes, rows, blocks) view and one copy brings all blocks
     uint32_t n_tiles;       // column tiles
@@ -240,6 +241,27 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
     // integer divisions) while the previous kernel may still be running
     GroupWalk<kBatched> walk(g);
     bool have = walk.next();       // the first group, too
+    // All weight blocks, once per CTA, on stage barrier 0: every CTA reads the same bytes, so
+    // they come out of L2 one reader after the other, and they are what the first tile waits
+    // for longest.  Block (tap, cb) = bytes [tap*C + cb*CB, +CB) of every filter lands in slot
+    // tap * c_blocks + cb.
+    auto issue_resident_weights = [&]() {
+        const uint32_t full = smem_u32(&bar_b_full[0]);
+        mbar_expect_tx(full, (uint32_t)kb_count * kBBlock);
+        if (g.w_one_copy) {
+            tma_load_3d(b_slot(0), &map_w, full, 0, 0, 0);
+        } else {
+            for (int kb = 0; kb < kb_count; ++kb) tma_load_2d(b_slot(kb), &map_w, full, kb * CB, 0);
+        }
+    };
+    // The weights are not an output of the kernel that runs before this one (the host checks
+    // that and sets early_weights), so their copy may start before that kernel has finished:
+    // in a chain of layers the wait for the weights then overlaps the predecessor's tail.
+    bool b_issued = false;
+    if (B_RESIDENT && g.early_weights && threadIdx.x == 0 && have) {
+        issue_resident_weights();
+        b_issued = true;
+    }
     dep_launch();
     dep_wait();
 
@@ -251,7 +273,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             uint32_t gi = 0;                   // group counter
             int rb = 0; uint32_t ruse = 0;     // its window buffer (gi % win_bufs) and that buffer's use count (gi / win_bufs)
             uint32_t it = 0;      // streamed weight-block counter
-            bool b_issued = false;  // resident weights requested
             long long pw = 0;
             const long long pt0 = SPARQ_PROF_NOW();
             for (; have; have = walk.next()) {
@@ -262,18 +283,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 const int oh0 = (int)walk.tin * g.TR;
                 if (gi == 0) SPARQ_PROF_STORE(9, SPARQ_PROF_NOW() - pt0);
                 if (B_RESIDENT && !b_issued) {
-                    // All weight blocks, once per CTA, on stage barrier 0, ahead of the first
-                    // window: every CTA reads the same bytes, so they come out of L2 one reader
-                    // after the other and are the last thing the first tile waits for.  Block
-                    // (tap, cb) = bytes [tap*C + cb*CB, +CB) of every filter lands in slot
-                    // tap * c_blocks + cb.
-                    const uint32_t full = smem_u32(&bar_b_full[0]);
-                    mbar_expect_tx(full, (uint32_t)kb_count * kBBlock);
-                    if (g.w_one_copy) {
-                        tma_load_3d(b_slot(0), &map_w, full, 0, 0, 0);
-                    } else {
-                        for (int kb = 0; kb < kb_count; ++kb) tma_load_2d(b_slot(kb), &map_w, full, kb * CB, 0);
-                    }
+                    issue_resident_weights();
                     b_issued = true;
                     SPARQ_PROF_STORE(14, SPARQ_PROF_NOW() - pt0);
                 }

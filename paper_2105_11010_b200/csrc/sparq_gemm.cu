@@ -209,6 +209,54 @@ static int pick_bn(int64_t M, int64_t N, int sms, bool transform)
     return best;
 }
 
+// ---- what the previous fused launch on a stream wrote ---------------------------------------------
+// The fused kernels are launched with programmatic stream serialization and let their successor
+// start early; a successor may fetch its WEIGHTS before it waits for them -- provided the weights
+// are not among their outputs.  Every fused launch records its output ranges per (device,
+// stream) here and learns whether its own weights are clear of the previous launch's.  Kernels
+// of other libraries never release their successor early, so only these launches matter.  A
+// stream that is not in the table (first launch, or evicted) counts as "not clear".
+struct LastLaunch {
+    bool used;
+    int dev;
+    cudaStream_t stream;
+    uint64_t age;
+    uintptr_t lo[3], hi[3];
+};
+constexpr int kLastSlots = 32;
+static LastLaunch g_last[kLastSlots];
+static uint64_t g_last_age = 0;
+static std::mutex g_last_mutex;
+
+static bool record_launch_weights_clear(cudaStream_t st, const sparq_epilogue *e, size_t out_elems, const void *wgt, size_t wgt_bytes)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return false; }
+    std::lock_guard<std::mutex> lock(g_last_mutex);
+    LastLaunch *slot = nullptr, *oldest = &g_last[0];
+    for (LastLaunch &l : g_last) {
+        if (l.used && l.dev == dev && l.stream == st) { slot = &l; break; }
+        if (!l.used || l.age < oldest->age || oldest->used && !l.used) oldest = &l;
+    }
+    bool clear = false;
+    if (slot) {
+        clear = true;
+        const uintptr_t w0 = (uintptr_t)wgt, w1 = w0 + wgt_bytes;
+        for (int i = 0; i < 3; ++i)
+            if (slot->lo[i] < w1 && w0 < slot->hi[i]) clear = false;
+    } else {
+        slot = oldest;
+    }
+    const void *outs[3] = {e->acc_out, e->f32_out, e->u8_out};
+    const size_t width[3] = {4, 4, 1};
+    slot->used = true; slot->dev = dev; slot->stream = st; slot->age = ++g_last_age;
+    for (int i = 0; i < 3; ++i) {
+        slot->lo[i] = (uintptr_t)outs[i];
+        slot->hi[i] = outs[i] ? (uintptr_t)outs[i] + out_elems * width[i] : 0;
+    }
+    return clear;
+}
+
 // Variant argument of the launchers: 4 = n = 4 with all five placements, 8 = another full
 // placement set (6opt, 7opt), 0 = the general kernels.
 static int variant_n(const XformArgs &x) { return x.widen_rounds != 0 ? 0 : (x.n == 4 ? 4 : 8); }
@@ -441,6 +489,7 @@ static int try_window_conv(const uint8_t *x_in, int n, int h, int w, int c, cons
     g.residual_scale = e->residual_scale;
     rc = next_transform_args(e, g.N, &g.next_mode, &g.next_rnd, &g.next_xf);
     if (rc != SPARQ_OK) return rc;
+    g.early_weights = record_launch_weights_clear(st, e, (size_t)n * ho * wo * (size_t)cout, wgt, (size_t)cout * (size_t)K) ? 1 : 0;
     cudaError_t ce;
     if (bn == 64) ce = launch_window_shape<64, 64, true>(mx, mx1, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
     else if (bn == 128 && resident) ce = launch_window_shape<128, 128, true>(mx, mx1, mw, g, x.mode, variant_n(x), x.rnd, grid, smem_bytes, st);
@@ -475,6 +524,7 @@ int gemm_with_status(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
     if (tiles >= ((int64_t)1 << 31)) return set_error(SPARQ_ERR_UNSUPPORTED, "more than 2^31 output tiles");
     const int grid = (int)(tiles < sms ? tiles : sms);
+    record_launch_weights_clear(st, e, (size_t)M * (size_t)N, B, (size_t)N * (size_t)ldb);
     cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
     if (ce != cudaSuccess) return cuda_error(ce, "sparq_gemm_kernel launch");
     return SPARQ_OK;
@@ -569,6 +619,7 @@ extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, in
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((cout + bn - 1) / bn);
     if (tiles >= ((int64_t)1 << 31)) return set_error(SPARQ_ERR_UNSUPPORTED, "more than 2^31 output tiles");
     const int grid = (int)(tiles < sms ? tiles : sms);
+    record_launch_weights_clear(st, e, (size_t)M * (size_t)cout, wgt, (size_t)cout * (size_t)K);
     cudaError_t ce = launch(bn, bk, ma, mb, g, x, grid, st);
     if (ce != cudaSuccess) return cuda_error(ce, "sparq_gemm_kernel (convolution) launch");
     return SPARQ_OK;
