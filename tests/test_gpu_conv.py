@@ -201,3 +201,32 @@ def test_rejected_arguments():
     big = torch.zeros((1, 12, 12, 16), dtype=torch.int32, device="cuda")
     with pytest.raises(sparq.SparqError):
         sparq.sparq_conv2d_nhwc_s8(x, w, (1, 1), (3, 3), sparq.SparqParams(), acc_out=big)   # pad >= filter
+
+
+def test_weights_written_by_the_previous_launch_are_not_fetched_early():
+    """Back-to-back fused launches overlap: a launch may fetch its weights while its predecessor
+    is still running -- unless the predecessor writes them.  Here the first convolution's
+    requantized output IS the second convolution's weight tensor (same bytes read as int8);
+    the second launch must see the finished values."""
+    c = 128
+    x1 = synth.activations(31, (1, 36, 32, c), 0.4)
+    w1 = synth.weights(31, (c, 3, 3, c))
+    scale1, bias1 = synth.scales(31, c), synth.bias(31, c)
+    inv1 = synth.inv_out_scale(9 * c, 0.4) * 2.0
+    x2 = synth.activations(32, (3, 28, 28, c), 0.5)
+    acc1 = oracle.conv2d_nhwc(x1, w1, (1, 1), (1, 1), *V5)
+    _, q1 = oracle.epilogue(acc1, scale1, bias1, True, inv1)
+    w2 = q1.reshape(-1).view(np.int8).reshape(c, 3, 3, c)             # 1152 pixels x 128 channels = 128 x 3 x 3 x 128 bytes
+    want = oracle.conv2d_nhwc(x2, w2, (1, 1), (1, 1), *V5)
+    p = sparq.SparqParams(*V5)
+    x1d, w1d, x2d = torch.from_numpy(x1).cuda(), torch.from_numpy(w1).cuda(), torch.from_numpy(x2).cuda()
+    s1, b1 = torch.from_numpy(scale1).cuda(), torch.from_numpy(bias1).cuda()
+    wbuf = torch.zeros(c * 9 * c, dtype=torch.uint8, device="cuda")
+    acc2 = torch.zeros((3, 28, 28, c), dtype=torch.int32, device="cuda")
+    for _ in range(20):
+        wbuf.zero_()
+        sparq.sparq_conv2d_nhwc_s8(x1d, w1d, (1, 1), (1, 1), p, scale=s1, bias=b1, relu=True, inv_out_scale=inv1,
+                                   u8_out=wbuf.view(1, 36, 32, c))
+        sparq.sparq_conv2d_nhwc_s8(x2d, wbuf.view(torch.int8).view(c, 3, 3, c), (1, 1), (1, 1), p, acc_out=acc2)
+        sparq.sparq_check()
+        assert np.array_equal(acc2.cpu().numpy(), want)
