@@ -48,7 +48,10 @@ MIN_TIMED_MS = 50.0                 # device time every reported figure is the m
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarized under
 # profiles/; None whenever the kernel has changed since its capture.
-TRAFFIC = {"head": None, "rn18": None, "layer1x1": None, "transform_per_2p28": 268445184 + 214811392}
+TRAFFIC = {"head": 13083392 + 0,                # profiles/sparq_conv_window_kernel_cfg5.txt (output still dirty in L2)
+           "rn18": None,
+           "layer1x1": 12931456 + 5281280,        # profiles/sparq_gemm_kernel_layer1x1.txt (mean of the two launches)
+           "transform_per_2p28": 268445184 + 214811392}   # profiles/quantize_vec_kernel_2p28.txt
 
 
 def ops_of(L):
@@ -166,8 +169,9 @@ class GraphTimer:
         torch.cuda.synchronize()
         self.replays = 0
 
-    def run(self, min_ms=MIN_TIMED_MS, barrier=None):
+    def run(self, min_ms=None, barrier=None):
         import torch
+        min_ms = MIN_TIMED_MS if min_ms is None else min(min_ms, MIN_TIMED_MS)
         probe0, probe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         probe0.record(); self.graph.replay(); probe1.record()
         torch.cuda.synchronize()
@@ -278,7 +282,7 @@ def roofline_tensor(ops, ms, mma, pk, clocks_mhz, traffic, kernel, alg_bytes):
 
 # ---- sections ------------------------------------------------------------------------------------
 
-def mma_peak_section(device, bns=(64, 128, 256), iters=4000):
+def mma_peak_section(device, bns=(64, 128, 256), iters=2000):
     """The tensor core's own rate: the library's MMA-only loop on every SM (operands resident in
     shared memory).  MAC/clk/SM from the slowest CTA's cycle count; TOP/s from CUDA events."""
     import torch
@@ -286,8 +290,7 @@ def mma_peak_section(device, bns=(64, 128, 256), iters=4000):
     cyc = torch.zeros(256, dtype=torch.int64, device=device)
     out = {}
     for bn in bns:
-        for _ in range(2):
-            sms = sparq.sparq_selftest_mma_rate(bn, iters, cyc)
+        sms = sparq.sparq_selftest_mma_rate(bn, iters, cyc)      # warm-up
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         e0.record()
@@ -600,6 +603,7 @@ SECTIONS = ["main", "transform", "pack", "frontend", "sparse24", "layer1x1", "mm
 
 
 def main():
+    global MIN_TIMED_MS
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
@@ -610,8 +614,11 @@ def main():
     ap.add_argument("--section", default="main", choices=SECTIONS,
                     help="print one section in full instead of the headline line (small runs for profiling)")
     ap.add_argument("--log2n", type=int, default=28, help="activations for the streaming sections (2^log2n)")
+    ap.add_argument("--min-ms", type=float, default=MIN_TIMED_MS,
+                    help="device time each graph-timed figure covers at least (lower it for profiler runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    MIN_TIMED_MS = args.min_ms
     if args.impl == "reference":
         run_reference(args)
         return
