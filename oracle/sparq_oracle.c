@@ -31,8 +31,8 @@
 
 /* ---- Section 3.1: bSPARQ ------------------------------------------------ */
 
-/* Index of the most significant set bit of a non-zero byte ("searching for the
- * first most significant toggled bit", Section 3.1). */
+/* Index of the most significant set bit of a non-zero byte (Section 3.1: the window
+ * is found by looking for the leading one). */
 static int leading_one(unsigned x)
 {
     int p = 7;
@@ -101,7 +101,8 @@ unsigned oracle_bsparq_window(unsigned x, int n, unsigned mask, int rnd, int *sh
 /* ---- Section 3.2: vSPARQ ------------------------------------------------ */
 
 /* A lone non-zero activation of a pair owns the whole 2n-bit budget (Section 1,
- * contributions; Section 5.1: "total window sizes are 6 and 4 bits" for n = 3, 2).
+ * contributions; Section 5.1 gives the pair's total window as 6 bits for n = 3 and 4 bits
+ * for n = 2).
  * With 2n >= 8 that is the exact 8-bit value.  Otherwise it is a 2n-bit window made
  * of the two adjacent n-bit halves of Eq. 4, which may sit at any shift 0..8-2n. */
 static unsigned lone_budget(unsigned x, int n, int rnd)
@@ -181,9 +182,9 @@ static int shift_rank(int s, unsigned mask)
 
 static int set_size(unsigned mask) { return shift_rank(5, mask); }
 
-/* The pair's metadata as ONE number ("grouping the metadata for several activations",
- * Section 5.1, is left open by the paper; this library groups the two ShiftCtrl fields and
- * the MuxCtrl of a pair): with ns allowed placements,
+/* The pair's metadata as ONE number (Section 5.1 mentions sharing metadata among several
+ * activations and leaves it open; this library groups the two ShiftCtrl fields and the
+ * MuxCtrl of a pair): with ns allowed placements,
  *   mux 0 -> id(opt1) * ns + id(opt2)      mux 1 -> ns*ns      mux 2 -> ns*ns + 1
  * so a pair has ns*ns + 2 states with vSPARQ and ns*ns without. */
 int oracle_pack_states(int mode, unsigned mask)
@@ -284,11 +285,11 @@ void oracle_gemm(const uint8_t *A, const int8_t *B, int32_t *acc,
 
 /* Weights pruned 2:4 are stored compressed: per output channel j and per group g of four
  * consecutive reduction indices, the two kept values vals[j][2g], vals[j][2g+1] and their
- * coordinates pos[j][2g] < pos[j][2g+1] in 0..3 (Section 4, "Only the non-zero-value
- * weights are stored with additional coordinates").  The coordinates pick two of the
- * group's four activations; vSPARQ then looks at THAT pair (Section 5.3: activations are
- * "first filtered through the multiplexers ... Then, vSPARQ comes into play, inspecting
- * pairs of activations"), so the transform depends on the output channel:
+ * coordinates pos[j][2g] < pos[j][2g+1] in 0..3 (Section 4: a sparse tensor core keeps the
+ * non-zero weights together with their coordinates).  The coordinates pick two of the
+ * group's four activations; vSPARQ then looks at THAT pair (Section 5.3: the activations
+ * pass the coordinate multiplexers first and are paired afterwards), so the transform
+ * depends on the output channel:
  *     acc[m][j] = sum_g  T2(A[m][4g+p0], A[m][4g+p1]) . (v0, v1)
  * with T2 the pair rule of Eq. 2 (mode 2), bSPARQ on each (mode 1) or the identity (mode 0).
  * K must be a multiple of 4.  Returns 0, or -1 for bad coordinates. */

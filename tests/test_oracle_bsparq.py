@@ -75,8 +75,8 @@ def test_named_sets_are_valid_and_region_counts():
 
 
 def test_window_follows_leading_one_full_set():
-    # "counting the leading zero bits": with every placement allowed the window's top
-    # bit is the leading one (or the window sits at the bottom for small values).
+    # Section 3.1 (the window position comes from the leading-zero count): with every placement
+    # allowed the window's top bit is the leading one (or the window sits at the bottom for small values).
     for n in (4, 3, 2):
         full = (1 << (9 - n)) - 1
         for x in range(1, 256):
