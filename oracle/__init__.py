@@ -62,6 +62,17 @@ def lib() -> ctypes.CDLL:
         L.oracle_pack.restype = i
         L.oracle_unpack.argtypes = [p, p, sz, sz, i, u, p]
         L.oracle_unpack.restype = i
+        L.oracle_pair_fields_n.argtypes = [u, u, i, i, u, i, ctypes.POINTER(u), ctypes.POINTER(i),
+                                           ctypes.POINTER(u), ctypes.POINTER(i), ctypes.POINTER(i)]
+        L.oracle_pair_fields_n.restype = None
+        L.oracle_pack_states_n.argtypes = [i, i, u]
+        L.oracle_pack_states_n.restype = i
+        L.oracle_pack_ctrl_bits_n.argtypes = [i, i, u]
+        L.oracle_pack_ctrl_bits_n.restype = i
+        L.oracle_pack_n.argtypes = [p, sz, sz, i, i, u, i, p, p]
+        L.oracle_pack_n.restype = i
+        L.oracle_unpack_n.argtypes = [p, p, sz, sz, i, i, u, p]
+        L.oracle_unpack_n.restype = i
         L.oracle_gemm.argtypes = [p, p, p, i64, i64, i64, i, i, u, i]
         L.oracle_gemm.restype = None
         L.oracle_gemm_sparse24.argtypes = [p, p, p, p, i64, i64, i64, i, i, u, i]
@@ -168,6 +179,48 @@ def unpack(data: np.ndarray, ctrl: np.ndarray, shape, mode: int, mask: int) -> n
     row_len = out.shape[-1]
     rows = out.size // row_len if row_len else 0
     if lib().oracle_unpack(_ptr(data), _ptr(ctrl), rows, row_len, mode, mask, _ptr(out)) != 0:
+        raise ValueError("row length must be a multiple of 16")
+    return out
+
+
+# ---- encoded form for any window width (Section 5.1) -------------------------------
+
+def pair_fields_n(a: int, b: int, mode: int, n: int, mask: int, rnd: int) -> Tuple[int, int, int, int, int]:
+    """(in1, opt1, in2, opt2, mux) for n-bit windows; a lone value is split into two n-bit halves."""
+    in1, in2 = ctypes.c_uint(0), ctypes.c_uint(0)
+    o1, o2, mux = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int(0)
+    lib().oracle_pair_fields_n(a, b, mode, n, mask, rnd, ctypes.byref(in1), ctypes.byref(o1),
+                               ctypes.byref(in2), ctypes.byref(o2), ctypes.byref(mux))
+    return int(in1.value), int(o1.value), int(in2.value), int(o2.value), int(mux.value)
+
+
+def pack_states_n(mode: int, n: int, mask: int) -> int:
+    return lib().oracle_pack_states_n(mode, n, mask)
+
+
+def pack_ctrl_bits_n(mode: int, n: int, mask: int) -> int:
+    return lib().oracle_pack_ctrl_bits_n(mode, n, mask)
+
+
+def pack_n(x: np.ndarray, mode: int, n: int, mask: int, rnd: int) -> Tuple[np.ndarray, np.ndarray]:
+    """(data plane, control plane) for n-bit windows: 2n data bytes and cb control bytes per 16 activations."""
+    x = _c(x, np.uint8)
+    row_len = x.shape[-1]
+    rows = x.size // row_len if row_len else 0
+    cb = pack_ctrl_bits_n(mode, n, mask)
+    data = np.empty(x.size // 16 * 2 * n, dtype=np.uint8)
+    ctrl = np.empty(x.size // 16 * cb, dtype=np.uint8)
+    if lib().oracle_pack_n(_ptr(x), rows, row_len, mode, n, mask, rnd, _ptr(data), _ptr(ctrl)) != 0:
+        raise ValueError("row length must be a multiple of 16")
+    return data, ctrl
+
+
+def unpack_n(data: np.ndarray, ctrl: np.ndarray, shape, mode: int, n: int, mask: int) -> np.ndarray:
+    data, ctrl = _c(data, np.uint8), _c(ctrl, np.uint8)
+    out = np.empty(shape, dtype=np.uint8)
+    row_len = out.shape[-1]
+    rows = out.size // row_len if row_len else 0
+    if lib().oracle_unpack_n(_ptr(data), _ptr(ctrl), rows, row_len, mode, n, mask, _ptr(out)) != 0:
         raise ValueError("row length must be a multiple of 16")
     return out
 

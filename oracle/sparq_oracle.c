@@ -255,6 +255,113 @@ int oracle_unpack(const uint8_t *data, const uint8_t *ctrl, size_t rows, size_t 
     return 0;
 }
 
+/* ---- the encoded form for any window width (Section 5.1: 3- and 2-bit windows) ------------ */
+
+/* Eq. 4's fields for n-bit windows.  Two non-zero activations: their n-bit windows and
+ * placements, as above.  A lone non-zero activation (vSPARQ) owns the pair's 2n-bit budget
+ * (Section 5.1: 6 bits for n = 3, 4 bits for n = 2): its 2n-bit window w at shift s_l in
+ * 0..8-2n is handed to the two multipliers as the two n-bit halves of Eq. 3 / Eq. 4,
+ *     in1 = w >> n at shift s_l + n,    in2 = w & (2^n - 1) at shift s_l,
+ * both against the lone activation's weight (mux 1: first slot, mux 2: second slot).
+ * For n = 4 the window is the whole byte at s_l = 0 and this is oracle_pair_fields. */
+void oracle_pair_fields_n(unsigned a, unsigned b, int mode, int n, unsigned mask, int rnd,
+                          unsigned *in1, int *opt1, unsigned *in2, int *opt2, int *mux)
+{
+    a &= 0xFFu; b &= 0xFFu;
+    if (mode == 2 && (b == 0 || a == 0)) {
+        unsigned x = (b == 0) ? a : b, w = x;
+        int sl = 0;
+        if (2 * n < 8) {
+            unsigned full = (1u << (8 - 2 * n + 1)) - 1u;      /* shifts 0 .. 8-2n */
+            w = oracle_bsparq_window(x, 2 * n, full, rnd, &sl);
+        }
+        *in1 = w >> n; *opt1 = sl + n;
+        *in2 = w & ((1u << n) - 1u); *opt2 = sl;
+        *mux = (b == 0) ? 1 : 2;
+    } else {
+        *in1 = oracle_bsparq_window(a, n, mask, rnd, opt1);
+        *in2 = oracle_bsparq_window(b, n, mask, rnd, opt2);
+        *mux = 0;
+    }
+}
+
+static int set_size_n(int n, unsigned mask) { return shift_rank(8 - n + 1, mask); }
+static int lone_places(int n) { return 8 - 2 * n + 1; }        /* n = 4: 1, n = 3: 3, n = 2: 5 */
+
+/* States of a pair: ns*ns for two windows; with vSPARQ also the lone window's placement in
+ * either slot: ns*ns + s_l (first slot), ns*ns + lone_places + s_l (second slot). */
+int oracle_pack_states_n(int mode, int n, unsigned mask)
+{
+    int ns = set_size_n(n, mask);
+    return ns * ns + (mode == 2 ? 2 * lone_places(n) : 0);
+}
+
+int oracle_pack_ctrl_bits_n(int mode, int n, unsigned mask)
+{
+    int states = oracle_pack_states_n(mode, n, mask), bits = 0;
+    while ((1 << bits) < states) ++bits;
+    return bits;
+}
+
+/* Packed stream for n-bit windows, per unit of 16 activations (8 pairs):
+ * data: pair j's field (in1 << n) | in2 at bits [j*2n, (j+1)*2n) of a little-endian integer
+ *       of 2n bytes (n = 4: one byte per pair, as oracle_pack);
+ * ctrl: pair j's state at bits [j*cb, (j+1)*cb) of a little-endian integer of cb bytes. */
+int oracle_pack_n(const uint8_t *in, size_t rows, size_t row_len, int mode, int n, unsigned mask, int rnd,
+                  uint8_t *data, uint8_t *ctrl)
+{
+    if (row_len % 16) return -1;
+    const int ns = set_size_n(n, mask), cb = oracle_pack_ctrl_bits_n(mode, n, mask), nl = lone_places(n);
+    for (size_t u = 0; u < rows * row_len / 16; ++u) {
+        uint64_t dword = 0, cword = 0;
+        for (int j = 0; j < 8; ++j) {
+            unsigned in1, in2;
+            int opt1, opt2, mux;
+            oracle_pair_fields_n(in[16 * u + 2 * j], in[16 * u + 2 * j + 1], mode, n, mask, rnd,
+                                 &in1, &opt1, &in2, &opt2, &mux);
+            dword |= (uint64_t)((in1 << n) | in2) << (j * 2 * n);
+            unsigned state = mux == 0 ? (unsigned)(shift_rank(opt1, mask) * ns + shift_rank(opt2, mask))
+                                      : (unsigned)(ns * ns + (mux - 1) * nl + opt2);
+            cword |= (uint64_t)state << (j * cb);
+        }
+        for (int k = 0; k < 2 * n; ++k) data[(size_t)(2 * n) * u + k] = (uint8_t)(dword >> (8 * k));
+        for (int k = 0; k < cb; ++k) ctrl[(size_t)cb * u + k] = (uint8_t)(cword >> (8 * k));
+    }
+    return 0;
+}
+
+/* T(x) back from the packed stream: 2^opt1 * in1 and 2^opt2 * in2 (Eq. 4 with unit weights);
+ * for a lone value the two halves add up in its slot. */
+int oracle_unpack_n(const uint8_t *data, const uint8_t *ctrl, size_t rows, size_t row_len,
+                    int mode, int n, unsigned mask, uint8_t *out)
+{
+    if (row_len % 16) return -1;
+    const int ns = set_size_n(n, mask), cb = oracle_pack_ctrl_bits_n(mode, n, mask), nl = lone_places(n);
+    int shift_of[8], r = 0;
+    for (int t = 0; t <= 8 - n; ++t) if ((mask >> t) & 1u) shift_of[r++] = t;
+    for (size_t u = 0; u < rows * row_len / 16; ++u) {
+        uint64_t dword = 0, cword = 0;
+        for (int k = 0; k < 2 * n; ++k) dword |= (uint64_t)data[(size_t)(2 * n) * u + k] << (8 * k);
+        for (int k = 0; k < cb; ++k) cword |= (uint64_t)ctrl[(size_t)cb * u + k] << (8 * k);
+        for (int j = 0; j < 8; ++j) {
+            unsigned state = (unsigned)((cword >> (j * cb)) & ((1u << cb) - 1u));
+            unsigned f = (unsigned)((dword >> (j * 2 * n)) & ((1u << (2 * n)) - 1u));
+            unsigned in1 = f >> n, in2 = f & ((1u << n) - 1u), qa, qb;
+            if (state < (unsigned)(ns * ns)) {
+                qa = in1 << shift_of[state / ns];
+                qb = in2 << shift_of[state % ns];
+            } else {
+                unsigned t = state - (unsigned)(ns * ns), sl = t % (unsigned)nl;
+                unsigned v = (in1 << (sl + n)) + (in2 << sl);
+                if (t / (unsigned)nl == 0) { qa = v; qb = 0; } else { qa = 0; qb = v; }
+            }
+            out[16 * u + 2 * j] = (uint8_t)qa;
+            out[16 * u + 2 * j + 1] = (uint8_t)qb;
+        }
+    }
+    return 0;
+}
+
 /* ---- Eq. 1: the dot product over the transformed activations ------------- */
 
 /* acc[m][j] = sum_k T(A)[m][k] * B[k][j]; A is M x K (row-major, u8), B is the

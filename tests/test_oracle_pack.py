@@ -125,3 +125,92 @@ def test_footprint():
 def test_rejects_ragged_rows():
     with pytest.raises(ValueError):
         oracle.pack(np.zeros((2, 24), dtype=np.uint8), 2, 0x1F, 1)
+
+
+# ---- any window width (Section 5.1: 3- and 2-bit windows) -----------------------------------
+
+COMBOS_N = [(4, 0x1F), (4, 0x15), (3, 0x3F), (3, 0x35), (3, 0x29), (2, 0x7F), (2, 0x55), (2, 0x6B)]
+
+
+@pytest.mark.parametrize("n,mask", COMBOS_N)
+@pytest.mark.parametrize("mode", [1, 2])
+@pytest.mark.parametrize("rnd", [0, 1])
+def test_eq4_for_any_width_reproduces_the_transformed_pair(n, mask, mode, rnd):
+    # Eq. 4 evaluated with plain integers: 2^opt1 * in1 * w_in1 + 2^opt2 * in2 * w_in2 with the
+    # multiplexers choosing the weights equals T(a) * w1 + T(b) * w2; a lone value arrives as the
+    # two adjacent n-bit halves of its 2n-bit window (opt1 = opt2 + n).
+    shifts = {s for s in range(9 - n) if (mask >> s) & 1}
+    for a in range(0, 256, 3 if n == 4 else 1):
+        for b in list(range(0, 256, 5)) + [0, 1, 255]:
+            in1, o1, in2, o2, mux = oracle.pair_fields_n(a, b, mode, n, mask, rnd)
+            assert 0 <= in1 < (1 << n) and 0 <= in2 < (1 << n)
+            if mode == 2:
+                qa, qb = oracle.vsparq_pair(a, b, n, mask, rnd)
+            else:
+                qa, qb = oracle.bsparq(a, n, mask, rnd), oracle.bsparq(b, n, mask, rnd)
+            if mux == 0:
+                assert o1 in shifts and o2 in shifts
+            else:
+                assert mode == 2 and o1 == o2 + n and 0 <= o2 <= 8 - 2 * n
+                assert (mux == 1) == (b == 0)
+            for w1, w2 in [(1, 0), (0, 1), (-128, 127), (37, -91)]:
+                wa, wb = {0: (w1, w2), 1: (w1, w1), 2: (w2, w2)}[mux]
+                assert (in1 << o1) * wa + (in2 << o2) * wb == qa * w1 + qb * w2, (a, b)
+            if n == 4:
+                assert (in1, o1, in2, o2, mux) == oracle.pair_fields(a, b, mode, mask, rnd)
+
+
+def test_state_counts_and_widths_for_narrow_windows():
+    # two windows: ns^2 placements; a lone value: its 2n-bit window sits at one of 9 - 2n shifts, in either slot
+    for n, mask in COMBOS_N:
+        ns = bin(mask).count("1")
+        assert oracle.pack_states_n(1, n, mask) == ns * ns
+        assert oracle.pack_states_n(2, n, mask) == ns * ns + 2 * (9 - 2 * n)
+        for mode in (1, 2):
+            cb = oracle.pack_ctrl_bits_n(mode, n, mask)
+            assert (1 << cb) >= oracle.pack_states_n(mode, n, mask) > (1 << (cb - 1))
+    # Section 5.1's full sets: 6opt and 7opt need 6 control bits per pair: 6 and 5 bits per activation
+    assert oracle.pack_ctrl_bits_n(2, 3, 0x3F) == 6 and oracle.pack_ctrl_bits_n(2, 2, 0x7F) == 6
+    assert (2 * 3 + 6) / 2 == 6 and (2 * 2 + 6) / 2 == 5
+    assert oracle.pack_ctrl_bits_n(2, 4, 0x1F) == oracle.pack_ctrl_bits(2, 0x1F)
+
+
+@pytest.mark.parametrize("n,mask", COMBOS_N)
+@pytest.mark.parametrize("mode", [1, 2])
+@pytest.mark.parametrize("rnd", [0, 1])
+def test_round_trip_for_any_width_equals_the_transform(n, mask, mode, rnd):
+    x = all_pairs()
+    data, ctrl = oracle.pack_n(x, mode, n, mask, rnd)
+    assert data.size == x.size // 16 * 2 * n
+    back = oracle.unpack_n(data, ctrl, x.shape, mode, n, mask)
+    assert np.array_equal(back, oracle.transform(x, mode, n, mask, rnd))
+    if n == 4:      # the same stream as the byte-per-pair form
+        d4, c4 = oracle.pack(x, mode, mask, rnd)
+        assert np.array_equal(data, d4) and np.array_equal(ctrl, c4)
+
+
+def test_stream_bytes_worked_out_by_hand_for_three_bit_windows():
+    # vSPARQ, n = 3, all six placements, rounding.  One unit of 16 activations = 8 pairs:
+    #   (0, 0)     lone, first slot, w = 0 at s_l = 0          field 0b000000  state 36 + 0
+    #   (200, 0)   lone: 200 = 0b11001000 -> 6-bit window 0b110010 at s_l = 2 (exact)
+    #                                                           field 0b110010  state 36 + 2
+    #   (0, 77)    lone, second slot: 77 = 0b1001101 -> shift 1: (77 + 1) >> 1 = 39 = 0b100111
+    #                                                           field 0b100111  state 36 + 3 + 1
+    #   (5, 3)     windows 5 (shift 0), 3 (shift 0)            field 0b101011  state 0
+    #   (27, 100)  27 = 0b11011 -> shift 2: (27 + 2) >> 2 = 7 ; 100 = 0b1100100 -> shift 4: (100 + 8) >> 4 = 6
+    #                                                           field 0b111110  state 2 * 6 + 4
+    #   (255, 255) saturate: 7 at shift 5 both                  field 0b111111  state 5 * 6 + 5
+    #   (31, 63)   31 -> shift 2: (31 + 2) >> 2 = 8 carries to 32 = 4 << 3 ; 63 -> shift 3: (63 + 4) >> 3 = 8 -> 64 = 4 << 4
+    #                                                           field 0b100100  state 3 * 6 + 4
+    #   (1, 1)     field 0b001001  state 0
+    x = np.array([[0, 0, 200, 0, 0, 77, 5, 3, 27, 100, 255, 255, 31, 63, 1, 1]], dtype=np.uint8)
+    fields = [0b000000, 0b110010, 0b100111, 0b101011, 0b111110, 0b111111, 0b100100, 0b001001]
+    states = [36, 38, 40, 0, 16, 35, 22, 0]
+    dword = sum(f << (6 * j) for j, f in enumerate(fields))
+    cword = sum(s << (6 * j) for j, s in enumerate(states))
+    data, ctrl = oracle.pack_n(x, 2, 3, 0x3F, 1)
+    assert list(data) == [(dword >> (8 * k)) & 0xFF for k in range(6)]
+    assert list(ctrl) == [(cword >> (8 * k)) & 0xFF for k in range(6)]
+    want = [0, 0, 200, 0, 0, 78, 5, 3, 28, 96, 224, 224, 32, 64, 1, 1]
+    assert list(oracle.unpack_n(data, ctrl, x.shape, 2, 3, 0x3F)[0]) == want
+    assert list(oracle.transform(x, 2, 3, 0x3F, 1)[0]) == want
