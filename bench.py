@@ -337,25 +337,29 @@ def transform_section(device, pk, n, steps, warmup):
 
 
 def pack_section(device, pk, n, steps, warmup):
-    """Packed stream codec on n uint8 activations (50 % zeros, rows of 1024), vSPARQ n = 4,
-    five placements, round to nearest.  Algorithmic bytes of either direction = n (raw or
-    unpacked activations) + n/2 (data plane) + n/16 * ctrl_bits (control plane)."""
+    """Packed stream codec on n uint8 activations (50 % zeros, rows of 1024), vSPARQ, round to
+    nearest, for 4-, 3- and 2-bit windows with their full placement sets.  Algorithmic bytes of
+    either direction = n (raw or unpacked activations) + n/16 * 2w (data plane) + n/16 * ctrl_bits
+    (control plane), w = window bits."""
     import torch
     import paper_2105_11010_b200 as sparq
     sync = torch.cuda.synchronize
     x = device_activations(device, (n // 1024, 1024), 0.5, 6)
-    p = sparq.SparqParams(sparq.MODE_VSPARQ, 4, sparq.SET_5OPT, sparq.ROUND_NEAREST)
-    cb = sparq.sparq_packed_ctrl_bits(p)
-    data = torch.empty(n // 2, dtype=torch.uint8, device=device)
-    ctrl = torch.empty(n // 16 * cb, dtype=torch.uint8, device=device)
     y = torch.empty_like(x)
-    nbytes = n + n // 2 + n // 16 * cb
-    out = {"activations": n, "ctrl_bits_per_pair": cb, "bits_per_activation": 4 + cb / 2}
-    for name, fn in (("pack", lambda i: sparq.sparq_pack(x, p, data, ctrl)),
-                     ("unpack", lambda i: sparq.sparq_unpack(data, ctrl, p, y))):
-        ms = time_region(fn, steps, warmup, sync) / steps
-        gbs = nbytes / ms / 1e6
-        out[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1), "frac_of_copy": round(gbs / pk["hbm"], 4)}
+    out = {"activations": n}
+    for w, mask in ((4, sparq.SET_5OPT), (3, sparq.SET_6OPT), (2, sparq.SET_7OPT)):
+        p = sparq.SparqParams(sparq.MODE_VSPARQ, w, mask, sparq.ROUND_NEAREST)
+        cb = sparq.sparq_packed_ctrl_bits(p)
+        data = torch.empty(n // 16 * 2 * w, dtype=torch.uint8, device=device)
+        ctrl = torch.empty(n // 16 * cb, dtype=torch.uint8, device=device)
+        nbytes = n + n // 16 * 2 * w + n // 16 * cb
+        res = {"ctrl_bits_per_pair": cb, "bits_per_activation": w + cb / 2}
+        for name, fn in (("pack", lambda i: sparq.sparq_pack(x, p, data, ctrl)),
+                         ("unpack", lambda i: sparq.sparq_unpack(data, ctrl, p, y))):
+            ms = time_region(fn, steps, warmup, sync) / steps
+            gbs = nbytes / ms / 1e6
+            res[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1), "frac_of_copy": round(gbs / pk["hbm"], 4)}
+        out[f"n{w}"] = res
     sparq.sparq_check()
     return out
 

@@ -220,9 +220,10 @@ SPARQ_API int sparq_gemm_s8_static(const uint8_t *A, int64_t lda, const int8_t *
 /* ---- Packed stream ------------------------------------------------------------------------
  * The encoded form that the multiplier of Eq. 4 consumes, as a storage / bandwidth format
  * for activations between layers (the paper names the metadata as the method's footprint
- * cost and leaves grouping it open, Sections 5.1 and 6).  Defined for window_bits = 4 and
- * mode BSPARQ or VSPARQ (else SPARQ_ERR_INVALID_ARG / SPARQ_ERR_UNSUPPORTED); row_len must
- * be a multiple of 16 and all pointers 16-byte aligned (else SPARQ_ERR_UNSUPPORTED).
+ * cost and leaves grouping it open, Sections 5.1 and 6).  Defined for mode BSPARQ or VSPARQ
+ * (else SPARQ_ERR_INVALID_ARG); row_len must be a multiple of 16 and all pointers 16-byte
+ * aligned (else SPARQ_ERR_UNSUPPORTED).  The description below is for window_bits = 4; the
+ * 3- and 2-bit forms follow it.
  *
  * A pair (2j, 2j+1) of a row becomes
  *   one data byte  (in1 << 4) | in2: the two 4-bit windows of bSPARQ(a), bSPARQ(b) when the
@@ -238,10 +239,17 @@ SPARQ_API int sparq_gemm_s8_static(const uint8_t *A, int64_t lda, const int8_t *
  *   data plane: rows * row_len / 2 bytes, pairs in order.
  *   ctrl plane: rows * row_len / 16 * cb bytes: per 16 activations the 8 states, pair j at
  *               bits [j*cb, (j+1)*cb) of a little-endian integer of cb bytes.
+ * For window_bits n = 3 or 2 (Section 5.1) the fields are n bits wide: per 16 activations the
+ * data plane holds 2n bytes, pair j's field (in1 << n) | in2 at bits [j*2n, (j+1)*2n) of a
+ * little-endian integer (rows * row_len / 16 * 2n bytes in all; n = 4 is the byte-per-pair
+ * form above).  A lone non-zero value owns the pair's 2n-bit window at a shift s_l in
+ * 0..8-2n and travels as that window's two n-bit halves; its states are ns*ns + s_l (second
+ * slot zero) and ns*ns + (9 - 2n) + s_l (first slot zero).  6opt and 7opt with VSPARQ take
+ * cb = 6: 6 and 5 bits per activation.
  * sparq_unpack returns T(x) exactly (what sparq_quantize writes), so a consumer may run
  * with mode NONE on the unpacked tensor.  rows == 0 or row_len == 0 is a no-op. */
 
-/* Control bits per pair (2..5), or a negative sparq_status. */
+/* Control bits per pair (2..6), or a negative sparq_status. */
 SPARQ_API int sparq_packed_ctrl_bits(const sparq_params *p);
 
 /* in: rows x row_len activations.  data, ctrl: the two planes (sizes above), caller-owned. */

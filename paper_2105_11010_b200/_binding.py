@@ -275,10 +275,10 @@ def _rows(t: torch.Tensor):
 
 def sparq_pack(inp: torch.Tensor, params: SparqParams, data: torch.Tensor, ctrl: torch.Tensor, stream=None) -> None:
     """Packed stream of ``inp`` (rows along the last axis) into the caller's ``data``
-    (numel / 2 bytes) and ``ctrl`` (numel / 16 * ctrl_bits bytes) planes."""
+    (numel / 16 * 2 * window_bits bytes) and ``ctrl`` (numel / 16 * ctrl_bits bytes) planes."""
     rows, row_len = _rows(inp)
     cb = sparq_packed_ctrl_bits(params)
-    if data.numel() < inp.numel() // 2 or ctrl.numel() < inp.numel() // 16 * cb:
+    if data.numel() < inp.numel() // 16 * 2 * params.window_bits or ctrl.numel() < inp.numel() // 16 * cb:
         raise ValueError("data / ctrl plane too small")
     p = params._c()
     _raise(load_library().sparq_pack(_dev(inp, torch.uint8, "inp"), rows, row_len, ctypes.byref(p),
@@ -290,7 +290,7 @@ def sparq_unpack(data: torch.Tensor, ctrl: torch.Tensor, params: SparqParams, ou
     """``out`` (rows along the last axis) = T(x) of the packed stream."""
     rows, row_len = _rows(out)
     cb = sparq_packed_ctrl_bits(params)
-    if data.numel() < out.numel() // 2 or ctrl.numel() < out.numel() // 16 * cb:
+    if data.numel() < out.numel() // 16 * 2 * params.window_bits or ctrl.numel() < out.numel() // 16 * cb:
         raise ValueError("data / ctrl plane too small")
     p = params._c()
     _raise(load_library().sparq_unpack(_dev(data, torch.uint8, "data"), _dev(ctrl, torch.uint8, "ctrl"),

@@ -20,6 +20,11 @@
 
 namespace sparq {
 
+// 3- and 2-bit windows: sparq_pack_narrow.cu
+int narrow_ctrl_bits(const XformArgs &x);
+int pack_narrow(const uint8_t *in, uint8_t *data, uint8_t *ctrl, size_t units, const XformArgs &x, cudaStream_t st);
+int unpack_narrow(const uint8_t *data, const uint8_t *ctrl, uint8_t *out, size_t units, const XformArgs &x, cudaStream_t st);
+
 namespace {
 
 constexpr int kThreads = 512;
@@ -274,13 +279,12 @@ int state_bits(int mode, uint32_t mask)
     return bits;
 }
 
-// Validates the parameters of the packed form: a SPARQ mode with 4-bit windows.
+// Validates the parameters of the packed form: a SPARQ mode.
 int check_pack_params(const sparq_params *p, XformArgs *x)
 {
     int rc = validate_params(p, x);
     if (rc != SPARQ_OK) return rc;
     if (x->mode == SPARQ_MODE_NONE) return set_error(SPARQ_ERR_INVALID_ARG, "the packed form needs mode BSPARQ or VSPARQ");
-    if (x->n != 4) return set_error(SPARQ_ERR_UNSUPPORTED, "the packed form is defined for 4-bit windows (window_bits = %d)", x->n);
     return SPARQ_OK;
 }
 
@@ -353,7 +357,7 @@ extern "C" int sparq_packed_ctrl_bits(const sparq_params *p)
     XformArgs x;
     int rc = check_pack_params(p, &x);
     if (rc != SPARQ_OK) return rc;
-    return state_bits(x.mode, x.mask);
+    return x.n == 4 ? state_bits(x.mode, x.mask) : narrow_ctrl_bits(x);
 }
 
 extern "C" int sparq_pack(const uint8_t *in, size_t rows, size_t row_len, const sparq_params *p,
@@ -365,6 +369,7 @@ extern "C" int sparq_pack(const uint8_t *in, size_t rows, size_t row_len, const 
     if (rows == 0 || row_len == 0) return SPARQ_OK;
     size_t units = 0;
     if ((rc = check_stream(in, data, ctrl, in, rows, row_len, &units)) != SPARQ_OK) return rc;
+    if (x.n != 4) return pack_narrow(in, data, ctrl, units, x, (cudaStream_t)stream);
     const int ns = set_size(x.mask);
     const int cb = state_bits(x.mode, x.mask);
     // window and placement of bSPARQ(v) for every byte value, from the packed transform
@@ -401,6 +406,7 @@ extern "C" int sparq_unpack(const uint8_t *data, const uint8_t *ctrl, size_t row
     if (rows == 0 || row_len == 0) return SPARQ_OK;
     size_t units = 0;
     if ((rc = check_stream(data, ctrl, out, out, rows, row_len, &units)) != SPARQ_OK) return rc;
+    if (x.n != 4) return unpack_narrow(data, ctrl, out, units, x, (cudaStream_t)stream);
     const int ns = set_size(x.mask);
     const int cb = state_bits(x.mode, x.mask);
     int shift_of[5], r = 0;

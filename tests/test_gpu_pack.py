@@ -77,9 +77,7 @@ def test_empty_and_rejected():
     with pytest.raises(sparq.SparqError) as ei:                     # row_len not a multiple of 16
         sparq.sparq_pack(x, p, big, big)
     assert ei.value.code == -2
-    with pytest.raises(sparq.SparqError) as ei:                     # 3-bit windows have no packed form
-        sparq.sparq_packed_ctrl_bits(sparq.SparqParams(sparq.MODE_VSPARQ, 3, 0x3F, 1))
-    assert ei.value.code == -2
+    assert sparq.sparq_packed_ctrl_bits(sparq.SparqParams(sparq.MODE_VSPARQ, 3, 0x3F, 1)) == 6
     with pytest.raises(sparq.SparqError) as ei:                     # nothing to pack without SPARQ
         sparq.sparq_packed_ctrl_bits(sparq.SparqParams(sparq.MODE_NONE))
     assert ei.value.code == -1
@@ -87,3 +85,49 @@ def test_empty_and_rejected():
     with pytest.raises(sparq.SparqError) as ei:                     # misaligned plane
         sparq.sparq_pack(x, p, big[1:], big)
     assert ei.value.code == -2
+
+
+# ---- 3- and 2-bit windows (Section 5.1) -------------------------------------------------------
+
+NARROW = [(3, 0x3F), (3, 0x35), (3, 0x29), (2, 0x7F), (2, 0x55), (2, 0x6B)]
+
+
+def run_n(x, params):
+    n = params.window_bits
+    cb = sparq.sparq_packed_ctrl_bits(params)
+    xg = torch.from_numpy(x).cuda()
+    data = torch.full((x.size // 16 * 2 * n + 16,), 0xAA, dtype=torch.uint8, device="cuda")
+    ctrl = torch.full((x.size // 16 * cb + 16,), 0xAA, dtype=torch.uint8, device="cuda")
+    out = torch.zeros_like(xg)
+    sparq.sparq_pack(xg, params, data, ctrl)
+    sparq.sparq_unpack(data, ctrl, params, out)
+    sparq.sparq_check()
+    nd, nc = x.size // 16 * 2 * n, x.size // 16 * cb
+    assert (data[nd:] == 0xAA).all() and (ctrl[nc:] == 0xAA).all()      # nothing written past the planes
+    return cb, data[:nd].cpu().numpy(), ctrl[:nc].cpu().numpy(), out.cpu().numpy()
+
+
+@pytest.mark.parametrize("n,mask", NARROW)
+@pytest.mark.parametrize("mode", [sparq.MODE_BSPARQ, sparq.MODE_VSPARQ])
+@pytest.mark.parametrize("rnd", [0, 1])
+def test_every_pair_narrow_windows(n, mask, mode, rnd):
+    a, b = np.meshgrid(np.arange(256, dtype=np.uint8), np.arange(256, dtype=np.uint8), indexing="ij")
+    x = np.ascontiguousarray(np.stack([a.ravel(), b.ravel()], axis=1).reshape(-1, 64))
+    p = sparq.SparqParams(mode, n, mask, rnd)
+    cb, data, ctrl, out = run_n(x, p)
+    assert cb == oracle.pack_ctrl_bits_n(mode, n, mask)
+    wd, wc = oracle.pack_n(x, mode, n, mask, rnd)
+    assert np.array_equal(data, wd)
+    assert np.array_equal(ctrl, wc)
+    assert np.array_equal(out, oracle.transform(x, mode, n, mask, rnd))
+
+
+@pytest.mark.parametrize("shape", [(1, 16), (3, 48), (1025, 16), (777, 1024 + 16)])
+@pytest.mark.parametrize("n,mask", [(3, 0x3F), (2, 0x7F)])
+def test_ragged_shapes_narrow_windows(shape, n, mask):
+    x = synth.activations(90 + shape[0] + n, shape, 0.5)
+    p = sparq.SparqParams(sparq.MODE_VSPARQ, n, mask, 1)
+    _, data, ctrl, out = run_n(x, p)
+    wd, wc = oracle.pack_n(x, p.mode, n, mask, 1)
+    assert np.array_equal(data, wd) and np.array_equal(ctrl, wc)
+    assert np.array_equal(out, oracle.transform(x, p.mode, n, mask, 1))
