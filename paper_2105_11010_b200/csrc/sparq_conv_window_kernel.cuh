@@ -178,7 +178,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     volatile uint32_t *abort_flag = &abort_word;
-    const long long cta_t0 = SPARQ_PROF_NOW();
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t win_bytes = (uint32_t)g.plane_bytes * (uint32_t)g.c_blocks;
@@ -265,7 +264,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
     dep_launch();
     dep_wait();
 
-    if (threadIdx.x == 0) SPARQ_PROF_STORE(15, SPARQ_PROF_NOW() - cta_t0);
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -273,19 +271,15 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             uint32_t gi = 0;                   // group counter
             int rb = 0; uint32_t ruse = 0;     // its window buffer (gi % win_bufs) and that buffer's use count (gi / win_bufs)
             uint32_t it = 0;      // streamed weight-block counter
-            long long pw = 0;
-            const long long pt0 = SPARQ_PROF_NOW();
             for (; have; have = walk.next()) {
                 const int b = rb;                 // window buffer of this group and how often it was used before
                 const uint32_t use = ruse;
-                if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_win_empty[b]), (use - 1) & 1, abort_flag, g.status, g.wait_limit));
+                if (use > 0) mbar_wait(smem_u32(&bar_win_empty[b]), (use - 1) & 1, abort_flag, g.status, g.wait_limit);
                 if (*abort_flag) break;
                 const int oh0 = (int)walk.tin * g.TR;
-                if (gi == 0) SPARQ_PROF_STORE(9, SPARQ_PROF_NOW() - pt0);
                 if (B_RESIDENT && !b_issued) {
                     issue_resident_weights();
                     b_issued = true;
-                    SPARQ_PROF_STORE(14, SPARQ_PROF_NOW() - pt0);
                 }
                 for (int j = 0; j < g.G; ++j) {
                     const uint32_t wfull = smem_u32(&bar_win_full[b * kMaxG + j]);
@@ -300,17 +294,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                         // parity of every barrier of the buffer advances once per use
                         mbar_arrive(wfull);
                     }
-                    if (gi == 0 && j == 0) SPARQ_PROF_STORE(13, SPARQ_PROF_NOW() - pt0);
                 }
-#ifdef SPARQ_PROF
-                if (gi == 0) {
-                    SPARQ_PROF_TL(3, 1, cta_t0);
-                    for (int j = 0; j < (int)walk.cnt; ++j) {
-                        mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), 0, abort_flag, g.status, g.wait_limit);
-                        SPARQ_PROF_TL(3, 2 + j, cta_t0);
-                    }
-                }
-#endif
                 ++gi;
                 if (++rb == g.win_bufs) { rb = 0; ++ruse; }
                 if (!B_RESIDENT) {
@@ -332,8 +316,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     if (stop) break;
                 }
             }
-            SPARQ_PROF_STORE(0, pw);
-            SPARQ_PROF_STORE(1, SPARQ_PROF_NOW() - pt0);
             if (*abort_flag) {
                 // wait (bounded) for copies still in flight so that none lands after exit
                 const uint32_t gfirst = gi > (uint32_t)g.win_bufs ? gi - g.win_bufs : 0;
@@ -370,14 +352,12 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
             uint32_t gi = 0;                   // group counter
             int rb = 0; uint32_t ruse = 0;     // its window buffer (gi % win_bufs) and that buffer's use count (gi / win_bufs)
             int s = 0;  uint32_t bph = 0;      // streamed weight stage and its phase parity
-            long long mw = 0, ma = 0, mb = 0, mi = 0;
-            const long long mt0 = SPARQ_PROF_NOW();
             // descriptor steps, in 16-byte units: one padded input row, one channel-block plane,
             // the rows of one tile
             const uint32_t row16 = (uint32_t)(g.Wp * CB) >> 4;
             const uint32_t plane16 = (uint32_t)g.plane_bytes >> 4;
             const uint32_t tile16 = (uint32_t)(g.TR * g.Wp * CB) >> 4;
-            if (B_RESIDENT) SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, g.wait_limit));
+            if (B_RESIDENT) mbar_wait(smem_u32(&bar_b_full[0]), 0, abort_flag, g.status, g.wait_limit);
             for (; have; have = walk.next()) {
                 const int b = rb;
                 const uint32_t wph = ruse & 1u;
@@ -399,15 +379,15 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                         issued = true;
                         for (int j = 0; j < cnt; ++j) {
                             const uint32_t t = wt + (uint32_t)j, use = t / (uint32_t)kAcc;
-                            if (use > 0) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[t & (uint32_t)(kAcc - 1)]), (use - 1) & 1, abort_flag, g.status, g.wait_limit));
+                            if (use > 0) mbar_wait(smem_u32(&bar_acc_empty[t & (uint32_t)(kAcc - 1)]), (use - 1) & 1, abort_flag, g.status, g.wait_limit);
                         }
                         // all pieces of the group: the transform warps finish them in order; without a
                         // transform the copies land in any order
                         if (MODE == SPARQ_MODE_NONE) {
                             for (int j = 0; j < cnt; ++j)
-                                SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), wph, abort_flag, g.status, g.wait_limit));
+                                mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), wph, abort_flag, g.status, g.wait_limit);
                         } else {
-                            SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b * kMaxG + cnt - 1]), wph, abort_flag, g.status, g.wait_limit));
+                            mbar_wait(smem_u32(&bar_win_xf[b * kMaxG + cnt - 1]), wph, abort_flag, g.status, g.wait_limit);
                         }
                         tc_fence_after();
                         uint64_t a_cb = a_grp;
@@ -415,7 +395,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                             uint64_t a_r = a_cb;
                             for (int r = 0; r < g.R; ++r, a_r += row16) {
                                 for (int sx = 0; sx < g.S; ++sx) {
-                                    SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status, g.wait_limit));
+                                    mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status, g.wait_limit);
                                     tc_fence_after();
                                     const uint64_t bdesc = b_desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kBBlock >> 4));
                                     const uint64_t a_tap = a_r + (uint64_t)(uint32_t)(sx * (CB >> 4));
@@ -451,17 +431,15 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     const uint32_t acc = wt & (uint32_t)(kAcc - 1);
                     const uint32_t acc_use = wt / (uint32_t)kAcc;
                     const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
-                    if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 0, cta_t0);
-                    if (acc_use > 0 && !pre_acc) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status, g.wait_limit));
-                    if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 1, cta_t0);
+                    if (acc_use > 0 && !pre_acc) mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status, g.wait_limit);
                     // Tile j reads pieces 0..j.  The transform warps finish pieces in order, so with
                     // a transform piece j's barrier covers the earlier ones.  Without one the copies
                     // land in any order: this issuer waits for pieces j-1 and j (its previous tile
                     // of the group, j-2, waited for the two before).
                     const uint32_t ops_bar = smem_u32(MODE == SPARQ_MODE_NONE ? &bar_win_full[b * kMaxG + j] : &bar_win_xf[b * kMaxG + j]);
                     if (!pre_ops) {
-                        if (MODE == SPARQ_MODE_NONE && j > 0) SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar - 8u, wph, abort_flag, g.status, g.wait_limit));
-                        SPARQ_PROF_WAIT(mw, mbar_wait(ops_bar, wph, abort_flag, g.status, g.wait_limit));
+                        if (MODE == SPARQ_MODE_NONE && j > 0) mbar_wait(ops_bar - 8u, wph, abort_flag, g.status, g.wait_limit);
+                        mbar_wait(ops_bar, wph, abort_flag, g.status, g.wait_limit);
                     }
                     tc_fence_after();
                     pre_acc = pre_ops = 0;
@@ -477,8 +455,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                         pre_ops = (MODE == SPARQ_MODE_NONE) ? (uint32_t)((m & 6u) == 6u) : (m >> 2);
                     };
                     const uint64_t a_desc0 = a_grp + (uint64_t)((uint32_t)j * tile16);
-                    const long long is0 = SPARQ_PROF_NOW();
-                    if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 2, cta_t0);
                     // One (tap, channel block) of the tile: wait for its weights when they are
                     // streamed, then CB / 32 MMAs.  The descriptors are sums of warp-uniform
                     // loop-carried values (no table, no division), so the address arithmetic of
@@ -488,7 +464,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                         if (B_RESIDENT) {
                             bdesc = b_desc0 + (uint64_t)(slot * (uint32_t)(kBBlock >> 4));
                         } else {
-                            SPARQ_PROF_WAIT(mb, mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status, g.wait_limit));
+                            mbar_wait(smem_u32(&bar_b_full[s]), bph, abort_flag, g.status, g.wait_limit);
                             tc_fence_after();
                             bdesc = b_desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kBBlock >> 4));
                         }
@@ -526,10 +502,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                             }
                         }
                     }
-                    mi += SPARQ_PROF_NOW() - is0;
-                    if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 3, cta_t0);
                     tc_commit_if(smem_u32(&bar_acc_full[acc]), elected);      // accumulator complete
-                    if (me == 0) SPARQ_PROF_TL(0, 5 * (wt >> 1) + 4, cta_t0);
                 }
                 // The buffer goes back to the producer once both issuers have arrived and their
                 // MMAs have retired.  With a transform, first make sure that every transform warp
@@ -537,7 +510,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 // last), so that none of them can still be waiting on a phase when the producer
                 // starts the next.
                 if (MODE != SPARQ_MODE_NONE && (int)walk.cnt < g.G)
-                    SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_win_xf[b * kMaxG + g.G - 1]), wph, abort_flag, g.status, g.wait_limit));
+                    mbar_wait(smem_u32(&bar_win_xf[b * kMaxG + g.G - 1]), wph, abort_flag, g.status, g.wait_limit);
                 if (issued) {
                     tc_commit_if(smem_u32(&bar_win_empty[b]), elected);
                 } else {
@@ -551,16 +524,10 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 if (++rb == g.win_bufs) { rb = 0; ++ruse; }
             }
             if (me == 0) {
-                SPARQ_PROF_STORE(2, mw);
-                SPARQ_PROF_STORE(3, ma);
-                SPARQ_PROF_STORE(11, mb);
-                SPARQ_PROF_STORE(12, mi);
-                SPARQ_PROF_STORE(4, SPARQ_PROF_NOW() - mt0);
             }
             // all tensor-core work of this CTA has retired before tensor memory is freed
             tc_commit_if(smem_u32(&bar_done), elected);
             mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, g.wait_limit, true);
-            if (me == 0) SPARQ_PROF_TL(0, 40, cta_t0);
         }
         __syncwarp();
     } else if (warp < kFirstEpiWarp + epi_warps(MODE)) {
@@ -578,8 +545,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
         const int tr = slot / g.Wp;
         const int ow = slot - tr * g.Wp;
         const bool slot_ok = (tr < g.TR) && (ow < g.Wo);
-        long long ew = 0;
-        const long long et0 = SPARQ_PROF_NOW();
         // 64-wide tiles have one column tile and 16 or 32 columns per warp.  When only the
         // requantized bytes are wanted (the form every layer of a network uses), the warp keeps
         // the scale and bias of its columns in registers for the whole launch -- shared-memory
@@ -599,7 +564,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     const int64_t row = ((int64_t)walk.img * g.Ho + oh) * g.Wo + ow;
                     const uint32_t acc = wt & (uint32_t)(kAcc - 1);
                     const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + (uint32_t)cbase;
-                    SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status, g.wait_limit));
+                    mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status, g.wait_limit);
                     tc_fence_after();
 #pragma unroll 1
                     for (int ch = 0; ch < kTeamCols / 32; ++ch) {
@@ -637,9 +602,8 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 const bool row_ok = slot_ok && (oh < g.Ho);
                 uint8_t *dst = g.u8_out + (((int64_t)walk.img * g.Ho + oh) * g.Wo + ow) * 64 + cbase;
                 const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + (uint32_t)cbase;
-                if (!pre_full) SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status, g.wait_limit));
+                if (!pre_full) mbar_wait(smem_u32(&bar_acc_full[acc]), (wt / (uint32_t)kAcc) & 1u, abort_flag, g.status, g.wait_limit);
                 tc_fence_after();
-                if (warp == kFirstEpiWarp && lane == 0) SPARQ_PROF_TL(1, 2 * wt, cta_t0);
                 pre_full = 0;
 #pragma unroll
                 for (int hh = 0; hh < kColsPerWarp / 16; ++hh) {
@@ -674,7 +638,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     if (ev.next_mode != SPARQ_MODE_NONE) next_xform_words(w, 4, ev.next_mode, ev.next_rnd, ev.next_xf);
                     *reinterpret_cast<uint4 *>(dst + hh * 16) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
-                if (warp == kFirstEpiWarp && lane == 0) SPARQ_PROF_TL(1, 2 * wt + 1, cta_t0);
               }
             }
         } else
@@ -687,7 +650,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 staged_nt = nt;
                 epi_stage_scale_bias<kEpi>(g, nt * BN, BN, et, s_scale, s_bias);
             }
-            SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status, g.wait_limit));
+            mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status, g.wait_limit);
             tc_fence_after();
             const int oh = ((int)walk.tin + j) * g.TR + tr;
             const bool row_ok = slot_ok && (oh < g.Ho);
@@ -699,8 +662,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
           }
         }
         if (warp == kFirstEpiWarp && lane == 0) {
-            SPARQ_PROF_STORE(5, ew);
-            SPARQ_PROF_STORE(6, SPARQ_PROF_NOW() - et0);
         }
     } else if (MODE != SPARQ_MODE_NONE) {
         // ================= transform: once per piece =================
@@ -709,14 +670,11 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
         const XformDev xf = g.xf;
         uint32_t gi = 0;
         int rb = 0; uint32_t ruse = 0;         // window buffer of the group (gi % win_bufs) and its use count (gi / win_bufs)
-        long long xw = 0;
-        const long long xt0 = SPARQ_PROF_NOW();
         for (; have; have = walk.next()) {
             const int b = rb;
             const uint32_t wph = ruse & 1u;
             for (int j = 0; j < g.G; ++j) {
-                SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), wph, abort_flag, g.status, g.wait_limit));
-                if (warp == kFirstXfWarp && lane == 0 && gi == 0) SPARQ_PROF_TL(2, 2 * j, cta_t0);
+                mbar_wait(smem_u32(&bar_win_full[b * kMaxG + j]), wph, abort_flag, g.status, g.wait_limit);
                 if (j < (int)walk.cnt) {
                     const uint32_t nvec = piece_len(j) >> 4;
                     uint32_t pbase = win_buf(b) + piece_off(j);
@@ -751,20 +709,16 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_win_xf[b * kMaxG + j]));
-                if (warp == kFirstXfWarp && lane == 0 && gi == 0) SPARQ_PROF_TL(2, 2 * j + 1, cta_t0);
             }
             ++gi;
                 if (++rb == g.win_bufs) { rb = 0; ++ruse; }
         }
         if (warp == kFirstXfWarp && lane == 0) {
-            SPARQ_PROF_STORE(7, xw);
-            SPARQ_PROF_STORE(8, SPARQ_PROF_NOW() - xt0);
         }
     }
 
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) { SPARQ_PROF_STORE(10, SPARQ_PROF_NOW() - cta_t0); SPARQ_PROF_TL(3, 0, cta_t0); }
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"

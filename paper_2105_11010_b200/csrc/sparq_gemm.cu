@@ -10,10 +10,6 @@
 
 namespace sparq {
 
-#ifdef SPARQ_PROF
-__device__ long long g_prof[148 * 16];
-__device__ long long g_prof_tl[4 * 64];
-#endif
 
 // Limit of the device-side waits of every fused launch, in SM cycles.
 static long long g_wait_limit = kWaitLimitCycles;
@@ -625,14 +621,3 @@ extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, in
     return SPARQ_OK;
 }
 
-#ifdef SPARQ_PROF
-// Profiling builds only: copies the per-CTA role counters of the last fused launch.
-extern "C" __attribute__((visibility("default"))) int sparq_prof_read(long long *out)
-{
-    return (int)cudaMemcpyFromSymbol(out, sparq::g_prof, sizeof(long long) * 148 * 16);
-}
-extern "C" __attribute__((visibility("default"))) int sparq_prof_read_timeline(long long *out)
-{
-    return (int)cudaMemcpyFromSymbol(out, sparq::g_prof_tl, sizeof(long long) * 4 * 64);
-}
-#endif

@@ -49,24 +49,6 @@ constexpr int kSmemBudget = 200 * 1024;  // for the stage ring
 // kernel argument, so that a diagnostic launch can make a wait run out in microseconds.
 constexpr long long kWaitLimitCycles = 2000000000LL;
 
-// Optional per-role cycle counters (builds with -DSPARQ_PROF -rdc=true only): how long each warp role
-// waited on its barriers and how long it ran, per CTA.  Compiled out otherwise.
-#ifdef SPARQ_PROF
-extern __device__ long long g_prof[148 * 16];
-#define SPARQ_PROF_NOW() clock64()
-#define SPARQ_PROF_STORE(slot, v) (g_prof[blockIdx.x * 16 + (slot)] = (v))
-extern __device__ long long g_prof_tl[4 * 64];      // CTA 0's timeline: [role][event]
-#define SPARQ_PROF_TL(role, idx, t0) do { if (blockIdx.x == 0 && (idx) < 64) g_prof_tl[(role) * 64 + (idx)] = clock64() - (t0); } while (0)
-#else
-#define SPARQ_PROF_TL(role, idx, t0) ((void)0)
-#define SPARQ_PROF_NOW() 0LL
-#define SPARQ_PROF_STORE(slot, v) ((void)(v))
-#endif
-#define SPARQ_PROF_WAIT(accum, stmt) do { const long long t_ = SPARQ_PROF_NOW(); stmt; accum += SPARQ_PROF_NOW() - t_; } while (0)
-// slots: 0 producer wait, 1 producer total, 2 MMA wait for operands, 3 MMA wait for a free
-// accumulator, 4 MMA total, 5 epilogue wait, 6 epilogue total, 7 transform wait,
-// 8 transform total, 10 CTA total, 11 MMA wait for weights, 12 MMA issue section
-
 struct GemmArgs {
     // problem
     int64_t M, N, K;        // GEMM view (K = r*s*c for the convolution)
@@ -706,7 +688,6 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     volatile uint32_t *abort_flag = &abort_word;
-    const long long cta_t0 = SPARQ_PROF_NOW();
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     auto a_stage = [&](int s) { return smem_base + (uint32_t)s * Cfg::kStageBytes; };
@@ -759,8 +740,6 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         // ================= TMA producer =================
         if (lane == 0) {
             uint32_t it = 0;   // running stage counter across tiles
-            long long pw = 0;
-            const long long pt0 = SPARQ_PROF_NOW();
             for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
                 const uint32_t mt = (n_tiles32 == 1) ? tile : tile / n_tiles32, nt = tile - mt * n_tiles32;
                 const int64_t m0 = (int64_t)mt * kBM;
@@ -776,7 +755,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 for (int kb = 0; kb < kb_count; ++kb, ++it) {
                     const int s = it % S;
                     const uint32_t use = it / S;
-                    if (use > 0) SPARQ_PROF_WAIT(pw, mbar_wait(smem_u32(&bar_empty[s]), (use - 1) & 1, abort_flag, g.status, g.wait_limit));
+                    if (use > 0) mbar_wait(smem_u32(&bar_empty[s]), (use - 1) & 1, abort_flag, g.status, g.wait_limit);
                     if (*abort_flag) break;   // stop issuing copies once the CTA has given up
                     const uint32_t full = smem_u32(&bar_full[s]);
                     mbar_expect_tx(full, Cfg::kStageBytes);
@@ -791,8 +770,6 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 }
                 if (*abort_flag) break;
             }
-            SPARQ_PROF_STORE(0, pw);
-            SPARQ_PROF_STORE(1, SPARQ_PROF_NOW() - pt0);
             // After an abort: wait (bounded) for the copies this thread still has in
             // flight, so that none lands after the CTA has exited.
             if (*abort_flag) {
@@ -815,17 +792,15 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             uint32_t local_tile = 0;
             int s = 0;             // stage
             uint32_t ph = 0;       // its phase parity
-            long long mw = 0, ma = 0;
-            const long long mt0 = SPARQ_PROF_NOW();
             for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
                 const int acc = local_tile & 1;
                 const uint32_t acc_use = local_tile >> 1;
-                if (acc_use > 0) SPARQ_PROF_WAIT(ma, mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status, g.wait_limit));
+                if (acc_use > 0) mbar_wait(smem_u32(&bar_acc_empty[acc]), (acc_use - 1) & 1, abort_flag, g.status, g.wait_limit);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 for (int kb = 0; kb < kb_count; ++kb) {
-                    if (MODE == SPARQ_MODE_NONE) SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_full[s]), ph, abort_flag, g.status, g.wait_limit));
-                    else SPARQ_PROF_WAIT(mw, mbar_wait(smem_u32(&bar_xf[s]), ph, abort_flag, g.status, g.wait_limit));
+                    if (MODE == SPARQ_MODE_NONE) mbar_wait(smem_u32(&bar_full[s]), ph, abort_flag, g.status, g.wait_limit);
+                    else mbar_wait(smem_u32(&bar_xf[s]), ph, abort_flag, g.status, g.wait_limit);
                     tc_fence_after();
                     const uint64_t st_off = (uint64_t)((uint32_t)s * (uint32_t)(Cfg::kStageBytes >> 4));
                     const uint64_t adesc = adesc0 + st_off, bdesc = bdesc0 + st_off;
@@ -838,9 +813,6 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 }
                 tc_commit_if(smem_u32(&bar_acc_full[acc]), elected);      // accumulator complete
             }
-            SPARQ_PROF_STORE(2, mw);
-            SPARQ_PROF_STORE(3, ma);
-            SPARQ_PROF_STORE(4, SPARQ_PROF_NOW() - mt0);
             // all tensor-core work of this CTA has retired before tensor memory is freed
             tc_commit_if(smem_u32(&bar_done), elected);
             mbar_wait(smem_u32(&bar_done), 0, abort_flag, g.status, g.wait_limit, true);
@@ -856,8 +828,6 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const EpiView ev = make_epi_view(g);
         uint32_t local_tile = 0;
         int64_t staged_nt = -1;
-        long long ew = 0;
-        const long long et0 = SPARQ_PROF_NOW();
         if (epi_teams) {
             constexpr int kTeamWarps = kEpi / 2;
             constexpr int kTeamCols = BN / (kTeamWarps / 4);          // columns per warp
@@ -869,7 +839,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 const int64_t row = (int64_t)tile * kBM + quarter * 32 + lane;    // one column tile: row tile = tile
                 const bool row_ok = row < g.M;
                 const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + team * BN + (uint32_t)tcbase;
-                SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[team]), (local_tile >> 1) & 1u, abort_flag, g.status, g.wait_limit));
+                mbar_wait(smem_u32(&bar_acc_full[team]), (local_tile >> 1) & 1u, abort_flag, g.status, g.wait_limit);
                 tc_fence_after();
 #pragma unroll 1
                 for (int ch = 0; ch < kTeamCols / 32; ++ch) {
@@ -897,7 +867,7 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 staged_nt = nt;
                 epi_stage_scale_bias<kEpi>(g, nt * BN, BN, et, s_scale, s_bias);
             }
-            SPARQ_PROF_WAIT(ew, mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status, g.wait_limit));
+            mbar_wait(smem_u32(&bar_acc_full[acc]), acc_use & 1, abort_flag, g.status, g.wait_limit);
             tc_fence_after();
             const int64_t row = mt * kBM + quarter * 32 + lane;
             const bool row_ok = row < g.M;
@@ -907,8 +877,6 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                                       smem_u32(&bar_acc_empty[acc]), lane);
         }
         if (warp == kFirstEpiWarp && lane == 0) {
-            SPARQ_PROF_STORE(5, ew);
-            SPARQ_PROF_STORE(6, SPARQ_PROF_NOW() - et0);
         }
     } else if (MODE != SPARQ_MODE_NONE) {
         // ================= transform =================
@@ -921,13 +889,11 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         static_assert(kVecs % kXfThreads == 0 && kPerThread % kBatch == 0, "A stage must split evenly over a team");
         const XformDev xf = g.xf;
         uint32_t it = 0;
-        long long xw = 0;
-        const long long xt0 = SPARQ_PROF_NOW();
         for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < kb_count; ++kb, ++it) {
                 if ((int)(it & 1u) != team) continue;      // the other team's stage
                 const int s = it % S;
-                SPARQ_PROF_WAIT(xw, mbar_wait(smem_u32(&bar_full[s]), (it / S) & 1, abort_flag, g.status, g.wait_limit));
+                mbar_wait(smem_u32(&bar_full[s]), (it / S) & 1, abort_flag, g.status, g.wait_limit);
                 const uint32_t base = a_stage(s) + (uint32_t)xt * 16u;
 #pragma unroll
                 for (int j0 = 0; j0 < kPerThread; j0 += kBatch) {
@@ -954,14 +920,11 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             }
         }
         if (warp == kFirstXfWarp && lane == 0) {
-            SPARQ_PROF_STORE(7, xw);
-            SPARQ_PROF_STORE(8, SPARQ_PROF_NOW() - xt0);
         }
     }
 
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) SPARQ_PROF_STORE(10, SPARQ_PROF_NOW() - cta_t0);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
