@@ -49,8 +49,8 @@ MIN_TIMED_MS = 50.0                 # device time every reported figure is the m
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarized under
 # profiles/; None whenever the kernel has changed since its capture.
 TRAFFIC = {"head": 13083392 + 0,                # profiles/sparq_conv_window_kernel_cfg5.txt (output still dirty in L2)
-           "rn18": None,
-           "layer1x1": 12931456 + 5281280,        # profiles/sparq_gemm_kernel_layer1x1.txt (mean of the two launches)
+           "rn18": 6541824 + 0,                  # profiles/sparq_conv_window_kernel_cfg2.txt
+           "layer1x1": 12931456 + 2238464,        # profiles/sparq_gemm_kernel_layer1x1.txt (mean of the two launches)
            "transform_per_2p28": 268445184 + 214811392}   # profiles/quantize_vec_kernel_2p28.txt
 
 
@@ -749,7 +749,8 @@ def main():
             rn = ConvLayer(device, RN18, sets=20, host_recipe=True)
             ms2, _, _ = GraphTimer(rn.fused(VS), args.steps, 3).run()
             r2 = roofline_tensor(ops_of(RN18), ms2, mma, pk, clocks["sm_mhz"], TRAFFIC["rn18"], "", sum(bytes_of(RN18)))
-            ex["cfg2_resnet18_conv"] = {"us": round(ms2 * 1e3, 2), "tops": r2["achieved"], "frac": r2["frac"]}
+            ex["cfg2_resnet18_conv"] = {"us": round(ms2 * 1e3, 2), "tops": r2["achieved"], "frac": r2["frac"],
+                                        "traffic": r2["traffic"]}
             del rn
             torch.cuda.empty_cache()
             ex["cfg3_resnet50_b64"] = sweep_section(device, pk, mma, clocks["sm_mhz"], 10, detail=args.full)
