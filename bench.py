@@ -272,10 +272,10 @@ def roofline_tensor(ops, ms, mma, pk, clocks_mhz, traffic, kernel, alg_bytes):
     return {
         "bound": "tensor", "achieved": round(tops, 1), "peak": round(peak, 1), "unit": "TOP/s",
         "frac": round(tops / peak, 4), "traffic": traffic,
-        "peak_source": (f"measured: own MMA-only kind::i8 loop, {mma['mac_per_clk_sm']:.0f} MAC/clk/SM x {mma['sms']} SMs x "
+        "peak_source": (f"measured: own MMA-only i8 loop, {mma['mac_per_clk_sm']:.0f} MAC/clk/SM x {mma['sms']} SMs x "
                         f"{clk:.0f} MHz sampled" if mma else f"{pk['source']} bf16 burst x 2"),
         "frac_of_nominal_4500": round(tops / NOMINAL_INT8_TOPS, 4),
-        "per": "step in a back-to-back stream, not an isolated launch",
+        "per": "step in a back-to-back stream",
         "kernel": kernel, "ops": ops, "bytes": alg_bytes,
     }
 
@@ -726,8 +726,8 @@ def main():
             "workload": "cfg5 conv3x3 128x28x28x128->128 s1 p1, fused vSPARQ n=4 5opt +R, 50% zeros, requant u8",
             "global_batch": L["nb"] * world,
             "l2": f"{layer.sets} rotating in/out sets, {layer.sets * (in_b + out_b) >> 20} MiB > 126 MiB L2",
-            "parallelism": f"replicas x{world}, no collective",
-            "timing": f"K steps per CUDA graph; median of {replays} replays ({timed_ms:.0f} ms)",
+            "parallelism": f"replicas x{world}",
+            "timing": f"median of {replays} graph replays of K steps ({timed_ms:.0f} ms)",
             "eager_ms_per_step": round(eager_ms_step, 5),
         },
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"]},
