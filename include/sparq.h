@@ -20,6 +20,13 @@
  *     sparq_gemm_s8_sparse24 -- may have enqueued their earlier kernels when a later launch
  *     fails; their outputs are then undefined).  No entry point throws, aborts or traps the
  *     device.
+ *   - Consecutive fused launches on one stream overlap at their edges (programmatic
+ *     dependent launch): a launch may set itself up, and fetch its WEIGHTS, while its
+ *     predecessor is finishing -- never its activations, scale, bias or residual.  The
+ *     library keeps, per device and stream, the output ranges of the last fused launch and
+ *     fetches weights early only when they are clear of them, so a layer whose weights the
+ *     previous layer has just written still sees the finished values; kernels of other
+ *     libraries never release their successor early.  Nothing for the caller to do.
  *   - The library is thread-compatible: concurrent calls are allowed, the error string
  *     is per host thread.
  */
