@@ -35,6 +35,7 @@ import sparq_synth as synth  # noqa: E402
 
 METRIC = "fused SPARQ INT8 conv TOPS"
 UNIT = "TOPS"
+WORKLOAD = "cfg5 conv3x3 128x28x28x128->128 s1 p1, fused vSPARQ n=4 5opt +R, 50% zeros, requant u8"
 
 # the layer the headline is quoted on (ablation config, fused vSPARQ 5opt +R, 50 % zeros)
 HEAD = dict(nb=128, h=28, w=28, c=128, cout=128, r=3, s=3, stride=1, pad=1, zf=0.5, seed=500)
@@ -595,7 +596,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": "ablation_conv3x3_b128_28x28x128_to_128_s1_p1 (CPU oracle, " + sample + ")"},
+        "config": {"workload": WORKLOAD, "sample": "CPU oracle, " + sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -723,7 +724,7 @@ def main():
         "warmup": args.warmup, "ms_per_step": round(ms_step, 6), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {
-            "workload": "cfg5 conv3x3 128x28x28x128->128 s1 p1, fused vSPARQ n=4 5opt +R, 50% zeros, requant u8",
+            "workload": WORKLOAD,
             "global_batch": L["nb"] * world,
             "l2": f"{layer.sets} rotating in/out sets, {layer.sets * (in_b + out_b) >> 20} MiB > 126 MiB L2",
             "parallelism": f"replicas x{world}",
