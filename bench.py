@@ -491,7 +491,7 @@ def cfg5_section(device, steps=20, warmup=3, full=True):
     return out
 
 
-def sweep_section(device, pk, mma, clk, steps=10, detail=False):
+def sweep_section(device, pk, mma, clk, steps=10, detail=False, only=None):
     """ResNet-50 sweep, batch 64, every conv shape (22 shapes, 52 instances), fused vSPARQ n = 4
     5opt +R with requantization.  Each layer against its own floor max(ops / tensor peak,
     bytes / measured copy bandwidth)."""
@@ -503,6 +503,8 @@ def sweep_section(device, pk, mma, clk, steps=10, detail=False):
     for li, S in enumerate(synth.resnet50_conv_layers()):
         zf = float(np.random.default_rng(100 + li).uniform(0.3, 0.7))
         L = dict(nb=64, h=S.h, w=S.w, c=S.cin, cout=S.cout, r=S.r, s=S.s, stride=S.stride, pad=S.pad, zf=zf, seed=100 + li)
+        if only and only not in f"{S.h}x{S.w}x{S.cin}->{S.cout} {S.r}x{S.s}/s{S.stride}":
+            continue
         layer = ConvLayer(device, L)
         ms, _, _ = GraphTimer(layer.fused(p), steps, 3).run(25.0)
         ops, nbytes = ops_of(L), sum(bytes_of(L))
@@ -619,6 +621,7 @@ def main():
     ap.add_argument("--section", default="main", choices=SECTIONS,
                     help="print one section in full instead of the headline line (small runs for profiling)")
     ap.add_argument("--log2n", type=int, default=28, help="activations for the streaming sections (2^log2n)")
+    ap.add_argument("--only", default=None, help="with --section sweep: only the layers whose name contains this text")
     ap.add_argument("--min-ms", type=float, default=MIN_TIMED_MS,
                     help="device time each graph-timed figure covers at least (lower it for profiler runs)")
     args = ap.parse_args()
@@ -668,7 +671,7 @@ def main():
         elif sec == "cfg5":
             res = cfg5_section(device, args.steps, args.warmup)
         elif sec == "sweep":
-            res = sweep_section(device, pk, mma_peak_section(device), None, args.steps, detail=True)
+            res = sweep_section(device, pk, mma_peak_section(device), None, args.steps, detail=True, only=args.only)
         else:   # cfg2
             layer = ConvLayer(device, RN18, sets=20, host_recipe=True)
             ms, _, _ = GraphTimer(layer.fused(VS), args.steps, args.warmup).run()
