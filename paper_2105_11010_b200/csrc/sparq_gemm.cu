@@ -504,7 +504,10 @@ int gemm_with_status(const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb
     int rc = device_info(&sms);
     if (rc != SPARQ_OK) return rc;
     const int64_t pad128 = (K + 127) / 128 * 128, pad64 = (K + 63) / 64 * 64;
-    const int bk = (pad64 < pad128) ? 64 : 128;   // the step that pads K the least; ties go to the wider one
+    // the step that pads K the least; ties go to the wider one -- and so does a long reduction whose
+    // padding stays below an eighth (K = 576: five 128-byte steps instead of nine 64-byte ones: each
+    // step is a hand-off between three warp roles, which is what a small launch is made of)
+    const int bk = (pad64 < pad128 && !(pad64 >= 320 && pad128 * 8 <= pad64 * 9)) ? 64 : 128;
     const int bn = pick_bn(M, N, sms, x.mode != SPARQ_MODE_NONE);
     CUtensorMap ma, mb;
     rc = encode_2d(&ma, A, K, M, lda, bk, kBM);
