@@ -661,8 +661,6 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                                       smem_u32(&bar_acc_empty[acc]), lane);
           }
         }
-        if (warp == kFirstEpiWarp && lane == 0) {
-        }
     } else if (MODE != SPARQ_MODE_NONE) {
         // ================= transform: once per piece =================
         const uint32_t xt = threadIdx.x - kFirstXfWarp * 32;
