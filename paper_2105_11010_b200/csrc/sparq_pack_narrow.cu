@@ -9,9 +9,12 @@
 //                pair's 2n-bit window at shift s_l in 0..8-2n and travels as its two n-bit
 //                halves: ns*ns + s_l in the first slot, ns*ns + (9 - 2n) + s_l in the second
 //
-// One thread owns one unit and computes the fields arithmetically from the packed transform
-// (no tables): these widths are the paper's secondary configurations, and the kernels are
-// plain streaming kernels.
+// One thread owns one unit: the packed transform first, then per value its placement from a
+// 256-entry shared-memory table (the bit scans that would compute it run in a slow pipe), and
+// per state its meaning from a 64-entry one on the way back.  A block's share of each plane is
+// put together in shared memory and moved as whole words.  These widths are the paper's
+// secondary configurations; the kernels are bound by their per-pair arithmetic and table
+// reads, not by memory.
 #include "sparq_common.cuh"
 
 namespace sparq {
