@@ -152,8 +152,9 @@ SPARQ_API int sparq_gemm_s8(const uint8_t *A, int64_t lda, const int8_t *B, int6
  * Output pixel (img, ho, wo) is row (img*Ho + ho)*Wo + wo of the M x cout outputs, with
  * Ho = (h + 2*pad_h - r)/stride_h + 1 and Wo likewise.
  * Requirements (else SPARQ_ERR_UNSUPPORTED): x and wgt 16-byte aligned, c a multiple of
- * 16 (of 64 unless the filter is 1x1 with unit stride and no padding), r, s in 1..7,
- * strides in 1..8, pads < filter size, r*s*c <= 65536. */
+ * 16 (a count that is not a multiple of 64 is read in 64-channel blocks whose tail is zero
+ * fill: correct, at the speed of the next multiple of 64), r, s in 1..7, strides in 1..8,
+ * pads < filter size, r*s*c <= 65536. */
 SPARQ_API int sparq_conv2d_nhwc_s8(const uint8_t *x, int n, int h, int w, int c,
                          const int8_t *wgt, int cout, int r, int s,
                          int stride_h, int stride_w, int pad_h, int pad_w,

@@ -586,7 +586,6 @@ extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, in
     if (r == 1 && s == 1 && stride_h == 1 && stride_w == 1 && pad_h == 0 && pad_w == 0)
         return gemm_impl(x_in, c, wgt, c, M, cout, c, x, e, st);
 
-    if (c % 64) return set_error(SPARQ_ERR_UNSUPPORTED, "c = %d must be a multiple of 64 for filters other than 1x1 stride 1", c);
     int sms = 0;
     rc = device_info(&sms);
     if (rc != SPARQ_OK) return rc;
@@ -607,9 +606,12 @@ extern "C" int sparq_conv2d_nhwc_s8(const uint8_t *x_in, int n, int h, int w, in
     GemmArgs g;
     memset(&g, 0, sizeof(g));
     g.M = M; g.N = cout; g.K = K;
-    g.k_blocks = (int)(K / bk);
+    // A channel count that is not a multiple of 64 takes a last block that reaches past C: the
+    // im2col copy fills those channels with zeros.
+    g.c_blocks = (c + bk - 1) / bk;
+    g.k_blocks = r * s * g.c_blocks;
     g.conv = 1;
-    g.c_blocks = c / bk;
+    g.tap_k = c;
     g.S = s;
     g.Ho = ho; g.Wo = wo;
     g.stride_h = stride_h; g.stride_w = stride_w; g.pad_h = pad_h; g.pad_w = pad_w;

@@ -55,7 +55,8 @@ struct GemmArgs {
     int k_blocks;           // number of BK-wide reduction steps
     // convolution geometry (conv = 1) for the im2col producer
     int conv;
-    int c_blocks;           // BK-wide channel blocks per filter tap
+    int c_blocks;           // BK-wide channel blocks per filter tap (the last one may reach past C: zero fill)
+    int tap_k;              // bytes of a filter row per tap (= C)
     int S;                  // filter width (taps are ordered r-major, s-minor)
     int Ho, Wo;
     int stride_h, stride_w, pad_h, pad_w;
@@ -759,14 +760,18 @@ sparq_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     if (*abort_flag) break;   // stop issuing copies once the CTA has given up
                     const uint32_t full = smem_u32(&bar_full[s]);
                     mbar_expect_tx(full, Cfg::kStageBytes);
+                    int bx = kb * BK;
                     if (g.conv) {
+                        // Channels past C arrive as zeros, so whatever the weight block holds
+                        // there (the next tap's first bytes) adds nothing.
                         const int tap = kb / g.c_blocks, cb = kb % g.c_blocks;
                         tma_load_im2col_4d(a_stage(s), &map_a, full, cb * BK, base_w, base_h, base_n,
                                            (uint16_t)(tap % g.S), (uint16_t)(tap / g.S));
+                        bx = tap * g.tap_k + cb * BK;
                     } else {
                         tma_load_2d(a_stage(s), &map_a, full, kb * BK, (int)m0);
                     }
-                    tma_load_2d(b_stage(s), &map_b, full, kb * BK, n0);
+                    tma_load_2d(b_stage(s), &map_b, full, bx, n0);
                 }
                 if (*abort_flag) break;
             }

@@ -191,12 +191,32 @@ def test_config5_ablation_fused_and_unfused(zero_frac):
         assert np.array_equal(fused.cpu().numpy().reshape(-1, cout)[pix], want), variant
 
 
+@pytest.mark.parametrize("cfg", [
+    # nb, h, w, c, cout, r, s, stride, pad: channel counts that are multiples of 16 but not of 64
+    (2, 9, 9, 16, 40, 3, 3, 1, 1),
+    (1, 12, 12, 48, 64, 3, 3, 2, 1),
+    (2, 10, 10, 160, 72, 5, 5, 1, 2),
+    (1, 8, 8, 96, 128, 7, 7, 1, 3),
+    (3, 11, 7, 32, 24, 1, 3, 1, 0),
+])
+@pytest.mark.parametrize("variant", [V5, (sparq.MODE_NONE, 4, 0x1F, 1), (sparq.MODE_VSPARQ, 2, 0x7F, 0)])
+def test_channel_counts_with_a_zero_filled_last_block(cfg, variant):
+    # the last 64-channel block of every tap reaches past c: those channels must count as zeros
+    # whatever the weights of the next tap are (dense random here)
+    nb, h, w, c, cout, r, s, stride, pad = cfg
+    x = synth.activations(sum(cfg), (nb, h, w, c), 0.2)
+    wt = synth.weights(sum(cfg), (cout, r, s, c))
+    check_full(x, wt, stride, pad, variant, seed=sum(cfg))
+
+
 def test_rejected_arguments():
     x = torch.zeros((1, 8, 8, 32), dtype=torch.uint8, device="cuda")
     w = torch.zeros((16, 3, 3, 32), dtype=torch.int8, device="cuda")
     acc = torch.zeros((1, 8, 8, 16), dtype=torch.int32, device="cuda")
     with pytest.raises(sparq.SparqError) as ei:
-        sparq.sparq_conv2d_nhwc_s8(x, w, (1, 1), (1, 1), sparq.SparqParams(), acc_out=acc)   # c % 64 for 3x3
+        sparq.sparq_conv2d_nhwc_s8(torch.zeros((1, 8, 8, 24), dtype=torch.uint8, device="cuda"),
+                                   torch.zeros((16, 3, 3, 24), dtype=torch.int8, device="cuda"),
+                                   (1, 1), (1, 1), sparq.SparqParams(), acc_out=acc)   # c % 16
     assert ei.value.code == -2
     big = torch.zeros((1, 12, 12, 16), dtype=torch.int32, device="cuda")
     with pytest.raises(sparq.SparqError):
