@@ -296,7 +296,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     }
                 }
                 ++gi;
-                if (++rb == g.win_bufs) { rb = 0; ++ruse; }
+            if (++rb == g.win_bufs) { rb = 0; ++ruse; }
                 if (!B_RESIDENT) {
                     bool stop = false;
                     const int passes = kBatched ? 1 : (int)walk.cnt;     // batched: one pass serves the whole group
@@ -521,9 +521,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     if (elected) mbar_arrive(smem_u32(&bar_win_empty[b]));
                 }
                 ++gi;
-                if (++rb == g.win_bufs) { rb = 0; ++ruse; }
-            }
-            if (me == 0) {
+            if (++rb == g.win_bufs) { rb = 0; ++ruse; }
             }
             // all tensor-core work of this CTA has retired before tensor memory is freed
             tc_commit_if(smem_u32(&bar_done), elected);
@@ -709,9 +707,7 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                 if (lane == 0) mbar_arrive(smem_u32(&bar_win_xf[b * kMaxG + j]));
             }
             ++gi;
-                if (++rb == g.win_bufs) { rb = 0; ++ruse; }
-        }
-        if (warp == kFirstXfWarp && lane == 0) {
+            if (++rb == g.win_bufs) { rb = 0; ++ruse; }
         }
     }
 

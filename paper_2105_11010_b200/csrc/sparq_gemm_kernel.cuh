@@ -328,15 +328,19 @@ __device__ __forceinline__ float dequant(int32_t acc, float scale, float bias, i
     return y;
 }
 
-// clamp(rint(y * inv_out_scale), 0, 255) without a float->int conversion: clamping to
-// [0, 255] first commutes with the rounding (both bounds are integers; NaN clamps to 0),
-// and adding 1.5 * 2^23 rounds to the nearest integer, ties to even, leaving that integer
-// in the low 8 bits of the float's bit pattern.
+// clamp(rint(y * inv_out_scale), 0, 255): one multiply and one saturating conversion (round
+// to nearest, ties to even; NaN gives 0).  The conversion runs in its own pipe; clamping and
+// rounding with fp32 instructions instead (max, min, add of 1.5 * 2^23) took three issue slots
+// of the pipes the rest of the epilogue is bound by.
+__device__ __forceinline__ uint32_t sat_u8_rn(float z)
+{
+    uint32_t u;
+    asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(u) : "f"(z));
+    return u;
+}
 __device__ __forceinline__ uint32_t requant_bits(float y, float inv_out_scale)
 {
-    float z = __fmul_rn(y, inv_out_scale);
-    z = fminf(fmaxf(z, 0.0f), 255.0f);
-    return __float_as_uint(__fadd_rn(z, 12582912.0f));
+    return sat_u8_rn(__fmul_rn(y, inv_out_scale));
 }
 
 // low bytes of four words -> one word
@@ -564,15 +568,14 @@ __device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c)
 
 // The form every layer of a network uses -- requantized bytes only, no residual, full 32-column
 // groups -- as straight-line code with nothing decided per element and the fp32 steps done two
-// columns at a time: per accumulator an exact int -> float step, one fma, one multiply, the
-// clamp and the rounding add, then three byte permutes per four columns.  Same IEEE sequence
-// per element as epi_chunk.
+// columns at a time: per accumulator an exact int -> float step, one fma, one multiply and the
+// saturating conversion, then three byte permutes per four columns.  Same IEEE sequence per
+// element as epi_chunk.
 template <bool SMALL>
 __device__ __forceinline__ void epi_chunk_u8(const EpiView &e, uint32_t (&v)[32], int64_t row, int64_t col0, int ct,
                                              const float *s_scale, const float *s_bias)
 {
     const uint64_t inv2 = f2_pack(e.inv_out_scale, e.inv_out_scale);
-    const uint64_t magic2 = f2_pack(12582912.0f, 12582912.0f);
     const uint64_t neg_magic2 = f2_pack(-12582912.0f, -12582912.0f);
     uint32_t w[8];
 #pragma unroll
@@ -589,12 +592,8 @@ __device__ __forceinline__ void epi_chunk_u8(const EpiView &e, uint32_t (&v)[32]
             const uint64_t y = f2_fma(t, h ? f2_pack(sc.z, sc.w) : f2_pack(sc.x, sc.y), h ? f2_pack(bi.z, bi.w) : f2_pack(bi.x, bi.y));
             float z0, z1;
             f2_unpack(f2_mul(y, inv2), z0, z1);
-            z0 = fminf(fmaxf(z0, 0.0f), 255.0f);
-            z1 = fminf(fmaxf(z1, 0.0f), 255.0f);
-            float r0, r1;
-            f2_unpack(f2_add(f2_pack(z0, z1), magic2), r0, r1);
-            b[2 * h] = __float_as_uint(r0);
-            b[2 * h + 1] = __float_as_uint(r1);
+            b[2 * h] = sat_u8_rn(z0);
+            b[2 * h + 1] = sat_u8_rn(z1);
         }
         w[q] = pack4(b[0], b[1], b[2], b[3]);
     }
