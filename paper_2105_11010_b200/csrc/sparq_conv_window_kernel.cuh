@@ -623,15 +623,15 @@ sparq_conv_window_kernel(const __grid_constant__ CUtensorMap map_x0, const __gri
                     uint32_t w[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        uint32_t bb[4];
+                        float z[4];
 #pragma unroll
                         for (int jj = 0; jj < 4; ++jj) {
                             const int c = hh * 16 + 4 * q + jj;
                             const float y = ev.small_acc ? dequant<true>((int32_t)v[4 * q + jj], rs[c], rb[c], ev.relu_op)
                                                          : dequant<false>((int32_t)v[4 * q + jj], rs[c], rb[c], ev.relu_op);
-                            bb[jj] = requant_bits(y, ev.inv_out_scale);
+                            z[jj] = __fmul_rn(y, ev.inv_out_scale);
                         }
-                        w[q] = pack4(bb[0], bb[1], bb[2], bb[3]);
+                        w[q] = requant_pack4(z[0], z[1], z[2], z[3]);
                     }
                     if (ev.next_mode != SPARQ_MODE_NONE) next_xform_words(w, 4, ev.next_mode, ev.next_rnd, ev.next_xf);
                     *reinterpret_cast<uint4 *>(dst + hh * 16) = make_uint4(w[0], w[1], w[2], w[3]);

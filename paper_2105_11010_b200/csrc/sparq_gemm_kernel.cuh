@@ -328,25 +328,17 @@ __device__ __forceinline__ float dequant(int32_t acc, float scale, float bias, i
     return y;
 }
 
-// clamp(rint(y * inv_out_scale), 0, 255): one multiply and one saturating conversion (round
-// to nearest, ties to even; NaN gives 0).  The conversion runs in its own pipe; clamping and
-// rounding with fp32 instructions instead (max, min, add of 1.5 * 2^23) took three issue slots
-// of the pipes the rest of the epilogue is bound by.
-__device__ __forceinline__ uint32_t sat_u8_rn(float z)
+// Four fp32 values on the output grid -> four bytes clamp(rint(z), 0, 255) in one word, z0 in
+// the low byte: a round-to-nearest-even conversion to int32 each (NaN gives 0, the infinities
+// the int32 limits), then two instructions that saturate two integers to bytes and pack them
+// beside the bytes already there.  Clamping and rounding with fp32 instructions (max, min, add
+// of 1.5 * 2^23) and permuting the bytes together took eleven issue slots where this takes six.
+__device__ __forceinline__ uint32_t requant_pack4(float z0, float z1, float z2, float z3)
 {
-    uint32_t u;
-    asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(u) : "f"(z));
-    return u;
-}
-__device__ __forceinline__ uint32_t requant_bits(float y, float inv_out_scale)
-{
-    return sat_u8_rn(__fmul_rn(y, inv_out_scale));
-}
-
-// low bytes of four words -> one word
-__device__ __forceinline__ uint32_t pack4(uint32_t a, uint32_t b, uint32_t c, uint32_t d)
-{
-    return prmt(prmt(a, b, 0x0040u), prmt(c, d, 0x0040u), 0x5410u);
+    uint32_t hi, w;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(__float2int_rn(z3)), "r"(__float2int_rn(z2)), "r"(0));
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(__float2int_rn(z1)), "r"(__float2int_rn(z0)), "r"(hi));
+    return w;
 }
 
 // The next layer's transform on requantized bytes (producer-side SPARQ): four adjacent output
@@ -510,10 +502,10 @@ __device__ __forceinline__ void epi_chunk(const EpiView &e, uint32_t (&v)[NV], i
         uint32_t w[NQ];
 #pragma unroll
         for (int q = 0; q < NQ; ++q)
-            w[q] = pack4(requant_bits(__uint_as_float(v[4 * q]), e.inv_out_scale),
-                         requant_bits(__uint_as_float(v[4 * q + 1]), e.inv_out_scale),
-                         requant_bits(__uint_as_float(v[4 * q + 2]), e.inv_out_scale),
-                         requant_bits(__uint_as_float(v[4 * q + 3]), e.inv_out_scale));
+            w[q] = requant_pack4(__fmul_rn(__uint_as_float(v[4 * q]), e.inv_out_scale),
+                                 __fmul_rn(__uint_as_float(v[4 * q + 1]), e.inv_out_scale),
+                                 __fmul_rn(__uint_as_float(v[4 * q + 2]), e.inv_out_scale),
+                                 __fmul_rn(__uint_as_float(v[4 * q + 3]), e.inv_out_scale));
         if (e.next_mode != SPARQ_MODE_NONE) next_xform_words(w, NQ, e.next_mode, e.next_rnd, e.next_xf);
         if (full) {
             if constexpr (NV == 32) {
@@ -569,8 +561,8 @@ __device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c)
 // The form every layer of a network uses -- requantized bytes only, no residual, full 32-column
 // groups -- as straight-line code with nothing decided per element and the fp32 steps done two
 // columns at a time: per accumulator an exact int -> float step, one fma, one multiply and the
-// saturating conversion, then three byte permutes per four columns.  Same IEEE sequence per
-// element as epi_chunk.
+// conversion back to an integer, then two saturating packs per four columns.  Same IEEE
+// sequence per element as epi_chunk.
 template <bool SMALL>
 __device__ __forceinline__ void epi_chunk_u8(const EpiView &e, uint32_t (&v)[32], int64_t row, int64_t col0, int ct,
                                              const float *s_scale, const float *s_bias)
@@ -582,7 +574,7 @@ __device__ __forceinline__ void epi_chunk_u8(const EpiView &e, uint32_t (&v)[32]
     for (int q = 0; q < 8; ++q) {
         const float4 sc = *reinterpret_cast<const float4 *>(&s_scale[ct + 4 * q]);
         const float4 bi = *reinterpret_cast<const float4 *>(&s_bias[ct + 4 * q]);
-        uint32_t b[4];
+        float z[4];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int32_t a0 = (int32_t)v[4 * q + 2 * h], a1 = (int32_t)v[4 * q + 2 * h + 1];
@@ -590,12 +582,9 @@ __device__ __forceinline__ void epi_chunk_u8(const EpiView &e, uint32_t (&v)[32]
             const uint64_t t = SMALL ? f2_add(f2_pack(__int_as_float(a0 + 0x4B400000), __int_as_float(a1 + 0x4B400000)), neg_magic2)
                                      : f2_pack(__int2float_rn(a0), __int2float_rn(a1));
             const uint64_t y = f2_fma(t, h ? f2_pack(sc.z, sc.w) : f2_pack(sc.x, sc.y), h ? f2_pack(bi.z, bi.w) : f2_pack(bi.x, bi.y));
-            float z0, z1;
-            f2_unpack(f2_mul(y, inv2), z0, z1);
-            b[2 * h] = sat_u8_rn(z0);
-            b[2 * h + 1] = sat_u8_rn(z1);
+            f2_unpack(f2_mul(y, inv2), z[2 * h], z[2 * h + 1]);
         }
-        w[q] = pack4(b[0], b[1], b[2], b[3]);
+        w[q] = requant_pack4(z[0], z[1], z[2], z[3]);
     }
     st_global_v8(e.u8_out + row * e.N + col0, w);
 }
