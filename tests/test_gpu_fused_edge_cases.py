@@ -219,6 +219,44 @@ def test_gemm_epilogue_ties_clamps_and_non_finite(K, N, mode, relu):
         assert np.array_equal(u8.cpu().numpy(), q_nb), (inv, "no bias")
 
 
+def float_bit_patterns(rng, n: int) -> np.ndarray:
+    """Floats drawn over the whole format: any sign, any exponent (subnormals, infinities and NaNs
+    included), plus a share near the output grid, where the rounding and the clamp decide."""
+    bits = rng.integers(0, 1 << 32, n, dtype=np.uint64).astype(np.uint32)
+    f = bits.view(F).copy()
+    near = rng.random(n) < 0.5
+    f[near] = (rng.integers(-600, 600, n)[near] / 2.0 + rng.choice([0.0, 1e-3, -1e-3, 2.0 ** -24], n)[near]).astype(F)
+    return f
+
+
+@pytest.mark.parametrize("K", [16, 144])                 # add-based and converted int -> float step
+@pytest.mark.parametrize("N", [64, 128, 256])
+@pytest.mark.parametrize("relu", [False, True])
+def test_requantization_over_arbitrary_float_bit_patterns(K, N, relu):
+    # the float -> byte step is a conversion followed by a saturating pack: every float the
+    # arithmetic before it can produce must come out as the oracle's clamp(rint(z), 0, 255)
+    rng = np.random.default_rng([K, N, int(relu)])
+    A, B = tie_problem(K, N, seed=3 * K + N)
+    acc = oracle.gemm(A, B, sparq.MODE_NONE, 4, 0x1F, 1)
+    Ad, Bd = torch.from_numpy(A).cuda(), torch.from_numpy(np.ascontiguousarray(B.T)).cuda()
+    p = sparq.SparqParams(sparq.MODE_NONE)
+    for rep in range(6):
+        scale, bias = float_bit_patterns(rng, N), float_bit_patterns(rng, N)
+        inv = float(float_bit_patterns(rng, 1)[0]) if rep else 1.0
+        f_want, q_want = oracle.epilogue(acc, scale, bias, relu, inv)
+        u8 = torch.full(acc.shape, 7, dtype=torch.uint8, device="cuda")
+        f32 = torch.full(acc.shape, -7.0, dtype=torch.float32, device="cuda")
+        sd, bd = torch.from_numpy(scale).cuda(), torch.from_numpy(bias).cuda()
+        sparq.sparq_gemm_s8(Ad, Bd, p, scale=sd, bias=bd, relu=relu, inv_out_scale=inv, u8_out=u8)
+        sparq.sparq_check()
+        assert np.array_equal(u8.cpu().numpy(), q_want), (rep, inv, "bytes only")
+        u8.fill_(7)
+        sparq.sparq_gemm_s8(Ad, Bd, p, scale=sd, bias=bd, relu=relu, inv_out_scale=inv, u8_out=u8, f32_out=f32)
+        sparq.sparq_check()
+        assert np.array_equal(u8.cpu().numpy(), q_want), (rep, inv, "with fp32")
+        assert same_floats(f32.cpu().numpy(), f_want), (rep, inv, "fp32")
+
+
 @pytest.mark.parametrize("K", [16, 144])
 @pytest.mark.parametrize("mode", [sparq.MODE_NONE, sparq.MODE_VSPARQ])
 def test_gemm_epilogue_edge_values_on_256_wide_tiles(K, mode):
